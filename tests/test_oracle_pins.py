@@ -1,0 +1,455 @@
+"""Pins for the fp64 CPU oracle: what the paper and the mathematics fix, independent of the oracle's own code.
+
+Each test is chosen so that a plausible mistake in the oracle (dropped term, wrong sign or index, transposed
+operand, wrong head-to-KV-head map, wrong tie rule) fails at least one of them.
+"""
+import itertools
+import math
+from fractions import Fraction
+from pathlib import Path
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2408_00167_b200 import workloads as wl
+
+GOLDEN = Path(__file__).resolve().parent / "golden"
+
+
+def _dense(rng, L, Hq, Hkv, nq, c, m, d, dtype="f32", cap=None):
+    """Single-request dense inputs in storage form."""
+    cap = c if cap is None else cap
+    q = wl.to_storage(rng.standard_normal((L, Hq, nq, d)), dtype)
+    ck = wl.to_storage(rng.standard_normal((L, Hkv, cap, d)), dtype)
+    hk = wl.to_storage(rng.standard_normal((L, Hkv, m, d)), dtype)
+    meta = dict(q_off=[0, nq], chunk_off=[0, m], cache_off=[0, cap], cache_len=[c])
+    return q, ck, hk, meta
+
+
+def _score(dtype, q, ck, hk, meta, Hq, Hkv, d, **kw):
+    return oracle.score(dtype, q, ck, hk, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, **meta, **kw)
+
+
+def _numpy_scores(q, ck, hk, c, Hq, Hkv, scale, group_mode=0):
+    """Textbook restatement with numpy: softmax(QK^T * scale) over keys, summed over prompt rows and group heads."""
+    qf, kf = q.astype(np.float64), np.concatenate([ck[:, :, :c], hk], axis=2).astype(np.float64)
+    g = Hq // Hkv
+    k_per_qhead = np.repeat(kf, g, axis=1)                       # query head h reads KV head h // g
+    s = np.einsum("lhpd,lhjd->lhpj", qf, k_per_qhead) * scale
+    s = s - s.max(axis=-1, keepdims=True)
+    w = np.exp(s)
+    w /= w.sum(axis=-1, keepdims=True)
+    per_head = w.sum(axis=2)                                     # [L][Hq][N]
+    if group_mode == 0:
+        return per_head.reshape(per_head.shape[0], Hkv, g, -1).sum(axis=2)
+    return per_head.sum(axis=1, keepdims=True)
+
+
+# ----------------------------------------------------------------------------- scoring
+
+def test_single_candidate_scores_group_rows():
+    # A key that is the only visible one gets softmax weight 1 from every row (Method, positional-bias paragraph).
+    rng = np.random.default_rng(1)
+    q, ck, hk, meta = _dense(rng, 2, 4, 2, 5, 0, 1, 8)
+    s = _score("f32", q, ck, hk, meta, 4, 2, 8)
+    assert s.shape == (2, 2, 1)
+    np.testing.assert_array_equal(s, np.full((2, 2, 1), 2 * 5.0))
+
+
+def test_two_candidates_logistic_closed_form():
+    rng = np.random.default_rng(2)
+    d, nq = 16, 3
+    q, ck, hk, meta = _dense(rng, 1, 1, 1, nq, 1, 1, d)
+    s = _score("f32", q, ck, hk, meta, 1, 1, d)[0, 0]
+    k0, k1 = ck[0, 0, 0].astype(np.float64), hk[0, 0, 0].astype(np.float64)
+    expect0 = sum(1.0 / (1.0 + math.exp(float(np.dot(q[0, 0, p].astype(np.float64), k1 - k0)) / math.sqrt(d)))
+                  for p in range(nq))
+    assert s[0] == pytest.approx(expect0, rel=1e-13)
+    assert s[1] == pytest.approx(nq - expect0, rel=1e-13)
+
+
+def test_uniform_when_keys_identical_or_queries_zero():
+    rng = np.random.default_rng(3)
+    L, Hq, Hkv, nq, c, m, d = 1, 4, 2, 3, 4, 5, 8
+    q, ck, hk, meta = _dense(rng, L, Hq, Hkv, nq, c, m, d)
+    ck[:] = ck[:, :, :1]
+    hk[:] = ck[:, :, :1]
+    s = _score("f32", q, ck, hk, meta, Hq, Hkv, d)
+    np.testing.assert_allclose(s, (Hq // Hkv) * nq / (c + m), rtol=1e-14)
+    q2, ck2, hk2, meta2 = _dense(rng, L, Hq, Hkv, nq, c, m, d)
+    q2[:] = 0
+    s2 = _score("f32", q2, ck2, hk2, meta2, Hq, Hkv, d)
+    np.testing.assert_allclose(s2, (Hq // Hkv) * nq / (c + m), rtol=1e-14)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("group_mode", [0, 1])
+def test_matches_numpy_restatement_and_rows_sum_to_one(dtype, group_mode):
+    rng = np.random.default_rng(4)
+    L, Hq, Hkv, nq, c, m, d, cap = 2, 6, 3, 7, 9, 6, 16, 12
+    q, ck, hk, meta = _dense(rng, L, Hq, Hkv, nq, c, m, d, dtype, cap=cap)
+    s = _score(dtype, q, ck, hk, meta, Hq, Hkv, d, group_mode=group_mode)
+    G = Hkv if group_mode == 0 else 1
+    assert s.shape == (L, G, cap + m)
+    ref = _numpy_scores(wl.from_storage(q, dtype), wl.from_storage(ck, dtype), wl.from_storage(hk, dtype),
+                        c, Hq, Hkv, 1 / math.sqrt(d), group_mode)
+    np.testing.assert_allclose(s[:, :, :c + m], ref, rtol=1e-12, atol=1e-15)
+    np.testing.assert_array_equal(s[:, :, c + m:], 0.0)            # capacity slack is left untouched
+    np.testing.assert_allclose(s.sum(axis=-1), (Hq // G) * nq, rtol=1e-13)   # softmax rows sum to 1
+
+
+def test_mpmath_second_opinion():
+    mp = pytest.importorskip("mpmath")
+    mp.mp.dps = 50
+    rng = np.random.default_rng(5)
+    Hq, Hkv, nq, c, m, d = 2, 1, 2, 2, 3, 4
+    q, ck, hk, meta = _dense(rng, 1, Hq, Hkv, nq, c, m, d)
+    q *= 6                                                       # peaked softmax: exercises the max-shift
+    s = _score("f32", q, ck, hk, meta, Hq, Hkv, d, scale=0.5)[0, 0]
+    keys = [ck[0, 0, j] for j in range(c)] + [hk[0, 0, j] for j in range(m)]
+    acc = [mp.mpf(0)] * (c + m)
+    for h in range(Hq):
+        for p in range(nq):
+            logits = [mp.mpf("0.5") * sum(mp.mpf(float(a)) * mp.mpf(float(b)) for a, b in zip(q[0, h, p], k))
+                      for k in keys]
+            Z = sum(mp.e ** x for x in logits)
+            acc = [a + mp.e ** x / Z for a, x in zip(acc, logits)]
+    for j in range(c + m):
+        assert float(abs(mp.mpf(float(s[j])) - acc[j]) / acc[j]) < 1e-13
+
+
+def test_shift_invariance_and_permutation_equivariance():
+    rng = np.random.default_rng(6)
+    L, Hq, Hkv, nq, c, m, d = 1, 4, 2, 5, 6, 7, 8
+    q, ck, hk, meta = _dense(rng, L, Hq, Hkv, nq, c, m, d)
+    base = _score("f32", q, ck, hk, meta, Hq, Hkv, d)
+    u = rng.integers(-2, 3, size=d).astype(np.float32)           # exactly representable shift
+    ck_i = np.round(ck * 4) / 4
+    hk_i = np.round(hk * 4) / 4
+    q_i = np.round(q * 4) / 4
+    s0 = _score("f32", q_i, ck_i, hk_i, meta, Hq, Hkv, d)
+    s1 = _score("f32", q_i, ck_i + u, hk_i + u, meta, Hq, Hkv, d)
+    np.testing.assert_allclose(s1, s0, rtol=1e-12)               # a per-row constant cancels in the softmax
+    perm = rng.permutation(c + m)
+    allk = np.concatenate([ck, hk], axis=2)[:, :, perm]
+    sp = _score("f32", q, np.ascontiguousarray(allk[:, :, :c]), np.ascontiguousarray(allk[:, :, c:]), meta,
+                Hq, Hkv, d)
+    np.testing.assert_allclose(sp, base[:, :, perm], rtol=1e-12)
+
+
+def test_gqa_head_mapping_is_block_not_interleaved():
+    # Only query heads 2,3 (KV head 1) see a distinguishing key; group 1 must react, group 0 must stay uniform.
+    d, nq, N = 8, 2, 4
+    q = np.zeros((1, 4, nq, d), np.float32)
+    q[0, 2:, :, 0] = 5.0
+    ck = np.zeros((1, 2, 0, d), np.float32)
+    hk = np.zeros((1, 2, N, d), np.float32)
+    hk[0, :, 1, 0] = 4.0
+    meta = dict(q_off=[0, nq], chunk_off=[0, N], cache_off=[0, 0], cache_len=[0])
+    s = _score("f32", q, ck, hk, meta, 4, 2, d)
+    np.testing.assert_allclose(s[0, 0], 2 * nq / N, rtol=1e-14)
+    assert s[0, 1, 1] > 0.99 * 2 * nq
+
+
+def test_row_lse_matches_definition():
+    rng = np.random.default_rng(7)
+    L, Hq, Hkv, nq, c, m, d = 1, 4, 2, 3, 2, 4, 8
+    q, ck, hk, meta = _dense(rng, L, Hq, Hkv, nq, c, m, d)
+    _, lse = _score("f32", q, ck, hk, meta, Hq, Hkv, d, want_lse=True)
+    kf = np.repeat(np.concatenate([ck, hk], axis=2).astype(np.float64), 2, axis=1)
+    logits = np.einsum("lhpd,lhjd->lhpj", q.astype(np.float64), kf) / math.sqrt(d)
+    np.testing.assert_allclose(lse, np.log(np.exp(logits).sum(-1)), rtol=1e-13)
+
+
+def test_bf16_widening_is_exact():
+    # 1.0 + 2^-7 is representable in bfloat16; the dot product must see exactly that value.
+    bits = np.array([[[[0x3F81]]]], dtype=np.uint16)              # q = 1.0078125
+    one = np.array([[[[0x3F80]]]], dtype=np.uint16)               # k = 1
+    two = np.array([[[[0x4000]]]], dtype=np.uint16)               # k = 2
+    meta = dict(q_off=[0, 1], chunk_off=[0, 1], cache_off=[0, 1], cache_len=[1])
+    s = oracle.score("bf16", bits, one, two, n_q_heads=1, n_kv_heads=1, head_dim=1, scale=1.0, **meta)[0, 0]
+    assert s[1] == pytest.approx(1 / (1 + math.exp(-1.0078125)), rel=1e-15)
+
+
+def test_normalisation_factor_is_rank_neutral():
+    # Prompt rows see every candidate, so count(A != 0)/(m + c) is the constant n_q (Method, bullet "Normalization").
+    rng = np.random.default_rng(8)
+    L, Hq, Hkv, nq, c, m, d = 1, 2, 1, 5, 4, 6, 8
+    q, ck, hk, meta = _dense(rng, L, Hq, Hkv, nq, c, m, d)
+    plain = _score("f32", q, ck, hk, meta, Hq, Hkv, d)
+    normed = _score("f32", q, ck, hk, meta, Hq, Hkv, d, apply_norm=True)
+    np.testing.assert_allclose(normed, plain * nq, rtol=1e-13)
+    for r in range(1, c + m):
+        np.testing.assert_array_equal(oracle.select_unit(plain[0, 0], r), oracle.select_unit(normed[0, 0], r))
+
+
+def test_ragged_batch_equals_separate_requests():
+    rng = np.random.default_rng(9)
+    L, Hq, Hkv, d = 2, 4, 2, 8
+    nqs, caps, lens, ms = [3, 1, 4], [5, 2, 6], [4, 0, 6], [3, 5, 0]
+    q_off, cache_off, chunk_off = wl.offsets(nqs), wl.offsets(caps), wl.offsets(ms)
+    q = rng.standard_normal((L, Hq, q_off[-1], d)).astype(np.float32)
+    ck = rng.standard_normal((L, Hkv, cache_off[-1], d)).astype(np.float32)
+    hk = rng.standard_normal((L, Hkv, chunk_off[-1], d)).astype(np.float32)
+    s = oracle.score("f32", q, ck, hk, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, q_off=q_off, chunk_off=chunk_off,
+                     cache_off=cache_off, cache_len=lens)
+    for b in range(3):
+        qb = np.ascontiguousarray(q[:, :, q_off[b]:q_off[b + 1]])
+        cb = np.ascontiguousarray(ck[:, :, cache_off[b]:cache_off[b] + lens[b]])
+        hb = np.ascontiguousarray(hk[:, :, chunk_off[b]:chunk_off[b + 1]])
+        sb = oracle.score("f32", qb, cb, hb, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, q_off=[0, nqs[b]],
+                          chunk_off=[0, ms[b]], cache_off=[0, lens[b]], cache_len=[lens[b]])
+        o = cache_off[b] + chunk_off[b]
+        np.testing.assert_array_equal(s[:, :, o:o + lens[b] + ms[b]], sb)
+
+
+# ----------------------------------------------------------------------------- selection
+
+def _brute_force_best_subset(scores, r):
+    """Exact arithmetic: among all r-subsets the maximum total score, ties -> lexicographically smallest indices."""
+    fr = [Fraction(float(x)) for x in scores]
+    best, best_sum = None, None
+    for sub in itertools.combinations(range(len(fr)), r):        # generated in lexicographic order
+        tot = sum(fr[i] for i in sub)
+        if best is None or tot > best_sum:
+            best, best_sum = sub, tot
+    return list(best)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_select_against_exhaustive_subsets(seed):
+    rng = np.random.default_rng(100 + seed)
+    N = int(rng.integers(1, 11))
+    levels = int(rng.integers(1, 5))
+    scores = rng.integers(0, levels, size=N).astype(np.float64) / 4 + (rng.random(N) if seed % 2 else 0.0)
+    for r in range(0, N + 3):
+        kept = oracle.select_unit(scores, r)
+        rr = min(r, N)
+        assert len(kept) == rr
+        assert np.all(np.diff(kept) > 0)
+        if 0 < rr:
+            assert kept.tolist() == _brute_force_best_subset(scores, rr)
+
+
+def test_select_budget_at_or_above_candidates_is_identity():
+    s = np.array([0.3, 0.1, 0.2, 0.9])
+    for r in (4, 5, 100):
+        np.testing.assert_array_equal(oracle.select_unit(s, r), np.arange(4))
+    assert len(oracle.select_unit(s, 0)) == 0
+    assert len(oracle.select_unit(np.zeros(0), 3)) == 0
+
+
+def test_select_ties_go_to_lower_position_and_nan_ranks_last():
+    np.testing.assert_array_equal(oracle.select_unit(np.array([1.0, 2.0, 1.0, 2.0, 1.0]), 3), [0, 1, 3])
+    np.testing.assert_array_equal(oracle.select_unit(np.array([np.nan, 0.0, np.nan, 0.0]), 2), [1, 3])
+    np.testing.assert_array_equal(oracle.select_unit(np.array([np.nan, -1.0, np.nan]), 2), [0, 1])
+    np.testing.assert_array_equal(oracle.select_unit(np.array([0.0, -0.0, 0.0]), 2), [0, 1])     # -0 == +0
+
+
+def test_huge_scale_gives_integer_argmax_counts():
+    # scale -> large turns each softmax row into an indicator of its arg-max key: scores are exact integers.
+    rng = np.random.default_rng(11)
+    Hq, Hkv, nq, c, m, d = 2, 1, 9, 3, 5, 4
+    q, ck, hk, meta = _dense(rng, 1, Hq, Hkv, nq, c, m, d)
+    s = _score("f32", q, ck, hk, meta, Hq, Hkv, d, scale=1e6)[0, 0]
+    keys = np.concatenate([ck, hk], axis=2)[0, 0].astype(np.float64)
+    counts = np.bincount(np.argmax(q[0].astype(np.float64).reshape(-1, d) @ keys.T, axis=1), minlength=c + m)
+    np.testing.assert_array_equal(s, counts.astype(np.float64))
+    kept = oracle.select_unit(s, 4)
+    order = sorted(range(c + m), key=lambda j: (-counts[j], j))[:4]
+    assert kept.tolist() == sorted(order)
+
+
+def test_paper_worked_cache_example():
+    txt = dict(line.split(":") for line in (GOLDEN / "cache_example.txt").read_text().splitlines()
+               if line and not line.startswith("#"))
+    positions = [int(x) for x in txt["cache_positions"].split()]
+    ranking = [int(x) for x in txt["ranking"].split()]
+    shifts = [int(x) for x in txt["shifts"].split()]
+    discarded = [int(x) for x in txt["discarded"].split()]
+    scores = np.zeros(len(positions))
+    for rank, tok in enumerate(ranking):
+        scores[positions.index(tok)] = 10.0 - rank               # any scores that realise the printed ranking
+    in_rank_order = oracle.select_unit(scores, len(ranking), rank_order=True)
+    assert in_rank_order.tolist() == ranking
+    assert [slot - tok for slot, tok in enumerate(in_rank_order.tolist())] == shifts
+    ascending = oracle.select_unit(scores, len(ranking))
+    assert ascending.tolist() == sorted(ranking)                 # same kept set, original order
+    assert sorted(set(positions) - set(ascending.tolist())) == discarded
+
+
+def test_batched_select_layout_and_budget_clamp():
+    rng = np.random.default_rng(12)
+    L, G = 2, 3
+    caps, lens, ms, budget = [4, 3], [2, 3], [3, 1], [4, 2]
+    cache_off, chunk_off = wl.offsets(caps), wl.offsets(ms)
+    scores = rng.random((L, G, cache_off[-1] + chunk_off[-1]))
+    kept, out_len = oracle.select(scores, chunk_off=chunk_off, cache_off=cache_off, cache_len=lens, budget=budget)
+    assert out_len.tolist() == [4, 2]
+    for l in range(L):
+        for g in range(G):
+            for b in range(2):
+                o = cache_off[b] + chunk_off[b]
+                N = lens[b] + ms[b]
+                want = oracle.select_unit(scores[l, g, o:o + N], budget[b])
+                got = kept[l, g, cache_off[b]:cache_off[b] + out_len[b]]
+                np.testing.assert_array_equal(got, want)
+                np.testing.assert_array_equal(kept[l, g, cache_off[b] + out_len[b]:cache_off[b + 1]], -1)
+
+
+# ----------------------------------------------------------------------------- compaction and the whole step
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("group_mode", [0, 1])
+def test_compact_is_a_bit_exact_gather(dtype, group_mode):
+    rng = np.random.default_rng(13)
+    L, Hkv, d = 2, 4, 8
+    G = Hkv if group_mode == 0 else 1
+    caps, lens, ms, budget = [6, 5], [4, 5], [3, 2], [5, 4]
+    cache_off, chunk_off = wl.offsets(caps), wl.offsets(ms)
+
+    def rnd(n):
+        a = rng.standard_normal((L, Hkv, n, d)).astype(np.float32)
+        return wl.to_storage(a, dtype)
+    ck, cv, hk, hv = rnd(cache_off[-1]), rnd(cache_off[-1]), rnd(chunk_off[-1]), rnd(chunk_off[-1])
+    cpos = rng.integers(0, 1000, size=(L, G, cache_off[-1])).astype(np.int32)
+    hpos = rng.integers(1000, 2000, size=chunk_off[-1]).astype(np.int32)
+    scores = rng.random((L, G, cache_off[-1] + chunk_off[-1]))
+    kept, out_len = oracle.select(scores, chunk_off=chunk_off, cache_off=cache_off, cache_len=lens, budget=budget)
+    ok, ov, op = oracle.compact(dtype, kept, out_len, ck, cv, cpos, hk, hv, hpos, n_kv_heads=Hkv, head_dim=d,
+                                group_mode=group_mode, chunk_off=chunk_off, cache_off=cache_off, cache_len=lens)
+    for l in range(L):
+        for h in range(Hkv):
+            g = h if group_mode == 0 else 0
+            for b in range(2):
+                cand_k = np.concatenate([ck[l, h, cache_off[b]:cache_off[b] + lens[b]],
+                                         hk[l, h, chunk_off[b]:chunk_off[b + 1]]])
+                cand_v = np.concatenate([cv[l, h, cache_off[b]:cache_off[b] + lens[b]],
+                                         hv[l, h, chunk_off[b]:chunk_off[b + 1]]])
+                cand_p = np.concatenate([cpos[l, g, cache_off[b]:cache_off[b] + lens[b]],
+                                         hpos[chunk_off[b]:chunk_off[b + 1]]])
+                idx = kept[l, g, cache_off[b]:cache_off[b] + out_len[b]]
+                sl = slice(cache_off[b], cache_off[b] + out_len[b])
+                np.testing.assert_array_equal(ok[l, h, sl], cand_k[idx])
+                np.testing.assert_array_equal(ov[l, h, sl], cand_v[idx])
+                np.testing.assert_array_equal(op[l, g, sl], cand_p[idx])
+
+
+def test_rescoring_a_kept_subset_equals_scoring_the_subset():
+    rng = np.random.default_rng(14)
+    Hq, Hkv, nq, c, m, d = 2, 1, 3, 5, 6, 8
+    q, ck, hk, meta = _dense(rng, 1, Hq, Hkv, nq, c, m, d)
+    s = _score("f32", q, ck, hk, meta, Hq, Hkv, d)
+    kept = oracle.select_unit(s[0, 0], 4)
+    allk = np.concatenate([ck, hk], axis=2)
+    sub = np.ascontiguousarray(allk[:, :, kept])
+    empty = np.zeros((1, Hkv, 0, d), np.float32)
+    s_sub = oracle.score("f32", q, sub, empty, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, q_off=[0, nq],
+                         chunk_off=[0, 0], cache_off=[0, 4], cache_len=[4])
+    ref = _numpy_scores(q, sub, empty, 4, Hq, Hkv, 1 / math.sqrt(d))
+    np.testing.assert_allclose(s_sub, ref, rtol=1e-12)
+
+
+def _run_document(cfg, layer, budgets_per_step=None):
+    """Drive the chunk loop of the Method section with the oracle for one layer; returns final positions per group."""
+    q = wl.prompt_q(cfg, layer)
+    B, Hkv, d = cfg.batch, cfg.n_kv_heads, cfg.head_dim
+    caps = [max(r.budget, 1) for r in cfg.requests] if budgets_per_step is None else \
+        [max(max(bs), 1) for bs in budgets_per_step]
+    cache_off = wl.offsets(caps)
+    ck = wl.to_storage(np.zeros((1, Hkv, cache_off[-1], d), np.float32), cfg.dtype)
+    cv = ck.copy()
+    cpos = np.full((1, cfg.n_groups, cache_off[-1]), -1, np.int32)
+    cache_len = np.zeros(B, np.int32)
+    planted_pos = [set() for _ in range(B)]
+    lens_seen = []
+    for step in range(cfg.n_steps):
+        ch = wl.chunk_kv(cfg, layer, step, q)
+        for b, r in enumerate(cfg.requests):
+            planted_pos[b] |= set((step * r.chunk + ch["planted"][b]).tolist())
+        budget = [r.budget for r in cfg.requests] if budgets_per_step is None else \
+            [bs[min(step, len(bs) - 1)] for bs in budgets_per_step]
+        out = oracle.step(cfg.dtype, wl.to_storage(q, cfg.dtype)[None], ck, cv, cpos,
+                          wl.to_storage(ch["k"], cfg.dtype)[None], wl.to_storage(ch["v"], cfg.dtype)[None],
+                          ch["chunk_pos"], n_q_heads=cfg.n_q_heads, n_kv_heads=Hkv, head_dim=d,
+                          group_mode=cfg.group_mode, q_off=wl.q_offsets(cfg), chunk_off=ch["chunk_off"],
+                          cache_off=cache_off, cache_len=cache_len, budget=budget, threads=4)
+        ck, cv, cpos, cache_len = out["out_k"], out["out_v"], out["out_pos"], out["out_len"]
+        lens_seen.append(cache_len.copy())
+    return cpos, cache_len, planted_pos, cache_off, lens_seen
+
+
+def test_planted_keys_survive_the_whole_document():
+    base = wl.CONFIGS["c2"]
+    cfg = wl.scaled(base, n_layers=1, n_q_heads=4, n_kv_heads=2, head_dim=32,
+                    requests=(wl.Request(8, 512, 64, 48), wl.Request(5, 200, 64, 32)), planted_frac=0.04)
+    cpos, cache_len, planted, cache_off, _ = _run_document(cfg, 0)
+    assert cache_len.tolist() == [48, 32]
+    for b in range(cfg.batch):
+        assert 0 < len(planted[b]) <= cfg.requests[b].budget // 2
+        for g in range(cfg.n_groups):
+            final = cpos[0, g, cache_off[b]:cache_off[b] + cache_len[b]]
+            assert np.all(np.diff(final) > 0)
+            assert planted[b] <= set(final.tolist())
+
+
+def test_paper_schedule_gives_linear_cache_growth():
+    # r_{it+1} = m/sigma + c_it with c_0 = 0 gives c_it = it*m/sigma and a final size k = n/sigma (Method; Table 1).
+    sigma, m, n = 4, 64, 512
+    k = n // sigma
+    steps = n // m
+    schedule = [min(k, (it + 1) * m // sigma) for it in range(steps)]
+    schedule[-1] = k
+    cfg = wl.scaled(wl.CONFIGS["c2"], n_layers=1, n_q_heads=2, n_kv_heads=1, head_dim=16,
+                    requests=(wl.Request(4, n, m, k),))
+    _, cache_len, _, _, lens_seen = _run_document(cfg, 0, budgets_per_step=[schedule])
+    assert [int(x[0]) for x in lens_seen] == [(it + 1) * m // sigma for it in range(steps)]
+    assert int(cache_len[0]) == k
+
+
+def test_step_equals_its_three_parts():
+    rng = np.random.default_rng(15)
+    st = wl.steady_state(wl.scaled(wl.CONFIGS["c4"], n_layers=1, n_q_heads=4, n_kv_heads=2, head_dim=16,
+                                   requests=(wl.Request(3, 64, 16, 8), wl.Request(6, 40, 16, 5))), [0])
+    kw = dict(n_kv_heads=2, head_dim=16)
+    meta = dict(chunk_off=st["chunk_off"], cache_off=st["cache_off"], cache_len=st["cache_len"])
+    out = oracle.step("bf16", st["q"], st["cache_k"], st["cache_v"], st["cache_pos"], st["chunk_k"], st["chunk_v"],
+                      st["chunk_pos"], n_q_heads=4, q_off=st["q_off"], budget=st["budget"], **kw, **meta)
+    s = oracle.score("bf16", st["q"], st["cache_k"], st["chunk_k"], n_q_heads=4, q_off=st["q_off"], **kw, **meta)
+    kept, out_len = oracle.select(s, budget=st["budget"], **meta)
+    ok, ov, op = oracle.compact("bf16", kept, out_len, st["cache_k"], st["cache_v"], st["cache_pos"], st["chunk_k"],
+                                st["chunk_v"], st["chunk_pos"], **kw, **meta)
+    np.testing.assert_array_equal(out["scores"], s)
+    np.testing.assert_array_equal(out["kept_idx"], kept)
+    np.testing.assert_array_equal(out["out_k"], ok)
+    np.testing.assert_array_equal(out["out_v"], ov)
+    np.testing.assert_array_equal(out["out_pos"], op)
+    del rng
+
+
+# ----------------------------------------------------------------------------- the input recipe
+
+@pytest.mark.parametrize("name,shrink", [("c1", {}),
+                                         ("c2", dict(n_layers=1, n_q_heads=4, n_kv_heads=4)),
+                                         ("c3", dict(n_layers=1, n_q_heads=8, n_kv_heads=2,
+                                                     requests=(wl.Request(128, 4096, 512, 512),))),
+                                         ("c5", dict(n_layers=1, n_q_heads=8, n_kv_heads=2,
+                                                     requests=(wl.Request(64, 8192, 512, 352),)))])
+def test_planted_keys_are_clear_top_scores(name, shrink):
+    cfg = wl.scaled(wl.CONFIGS[name], **shrink)
+    st = wl.steady_state(cfg, [0])
+    s = oracle.score(cfg.dtype, st["q"], st["cache_k"], st["chunk_k"], n_q_heads=cfg.n_q_heads,
+                     n_kv_heads=cfg.n_kv_heads, head_dim=cfg.head_dim, q_off=st["q_off"], chunk_off=st["chunk_off"],
+                     cache_off=st["cache_off"], cache_len=st["cache_len"], threads=8)
+    planted = st["planted"][0]
+    assert len(planted) > 0
+    mask = np.zeros(s.shape[-1], bool)
+    mask[planted] = True
+    for g in range(cfg.n_groups):
+        if cfg.dist == "normal":
+            assert s[0, g, mask].min() >= 2.0 * s[0, g, ~mask].max()
+        else:
+            # heavy-tailed keys: an outlier may outscore a planted key, but every planted key is retained
+            kept = oracle.select_unit(s[0, g, :int(st["cache_len"][0] + st["chunk_off"][1])], int(st["budget"][0]))
+            assert set(planted.tolist()) <= set(kept.tolist())
