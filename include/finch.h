@@ -1,0 +1,178 @@
+/*
+ * finch.h -- C ABI of the B200 (sm_100a) library for Finch's prompt-guided KV-cache
+ * compression step (arXiv 2408.00167, Section "Method").
+ *
+ * Problem statement (Section "Problem Formulation"): given a prompt and a long text
+ * processed chunk by chunk, keep in a fixed-size KV cache only the key/value pairs
+ * that are most relevant to the prompt.  One *step* takes the compressed cache so
+ * far plus the new chunk (together: the N = c + m candidates), scores every
+ * candidate by the attention the prompt's query rows give it, keeps the top-r
+ * candidates per layer and selection group, and writes their K/V rows, in original
+ * order, into the next cache.
+ *
+ * Conventions common to every call
+ * --------------------------------
+ *  - All tensor pointers are DEVICE pointers unless a parameter says "host".
+ *    The caller owns every buffer, including the workspace; the library allocates
+ *    only the context and one 4-byte device status word and frees only those.
+ *  - Work is enqueued asynchronously on `cuda_stream` (a cudaStream_t passed as
+ *    void*; NULL = the legacy default stream).  No call synchronises except
+ *    finch_device_status.
+ *  - Arguments are validated on the host; a call that returns anything but FINCH_OK
+ *    has enqueued nothing.  Nothing throws or aborts across this boundary.  Kernels
+ *    never trap: device-side anomalies (inconsistent batch metadata, a bounded wait
+ *    that ran out) set bits in the status word, read with finch_device_status.
+ *  - A context is bound to one device and is not thread-safe; use it from one host
+ *    thread and one stream at a time.
+ *  - There is no CPU fallback.  finch_ctx_create fails with FINCH_ERR_UNSUPPORTED on a
+ *    device that is not compute capability 10.x.  A context created with device < 0 is
+ *    validation-only: every call checks its arguments exactly as usual, then returns
+ *    FINCH_ERR_UNSUPPORTED instead of enqueuing work (finch_workspace_bytes still works).
+ *
+ * Layouts
+ * -------
+ *  A finch_tensor views [n_layers][heads][tokens][head_dim] with head_dim contiguous
+ *  and the three outer strides given in ELEMENTS.  Base pointer and every stride
+ *  times the element size must be multiples of 16 bytes.
+ *
+ *  Batches are packed along the token axis ("cu_seqlens" style), with three offset
+ *  arrays of batch+1 int32 each (device memory):
+ *     prompt_q        heads = n_q_heads,  request b owns token rows [q_off[b], q_off[b+1])
+ *     chunk_k/chunk_v heads = n_kv_heads, request b owns rows [chunk_off[b], chunk_off[b+1])
+ *     cache_*, out_*  heads = n_kv_heads, request b owns a region of CAPACITY
+ *                     cache_off[b+1]-cache_off[b] rows starting at cache_off[b], of which the first
+ *                     cache_len[b] (input) or out_len[b] (output) rows are valid
+ *  Candidate j of request b is cache row j for j < cache_len[b], else chunk row j - cache_len[b]
+ *  (Method, bullet "Extract prompt-guided submatrix": columns 1..m+c).  N_b = cache_len[b] + chunk_len[b].
+ *
+ *  Selection groups: G = n_kv_heads groups per layer in FINCH_GROUP_PER_KV_HEAD mode (a group sums the
+ *  n_q_heads/n_kv_heads query heads that share one KV head) or G = 1 in FINCH_GROUP_PER_LAYER mode (the paper's
+ *  sum over all H heads; the one index list then applies to every KV head of the layer).
+ *     scores    float32 [n_layers][G][total_cache + total_chunk], request b at cache_off[b] + chunk_off[b], N_b valid
+ *     kept_idx  int32   [n_layers][G][total_cache],               request b at cache_off[b], out_len[b] valid
+ *     cache_pos / out_pos int32 [n_layers][G][total_cache]  original token position of each cached row
+ *     chunk_pos int32   [total_chunk]                       original token position of each chunk row
+ *     row_lse   float32 [n_layers][n_q_heads][total_q]      natural-log sum-exp of each prompt row's logits
+ */
+#ifndef FINCH_H_
+#define FINCH_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct finch_ctx finch_ctx; /* opaque */
+
+typedef enum {
+    FINCH_OK = 0,
+    FINCH_ERR_INVALID_ARG = 1,         /* null pointer, negative size, overlap of outputs with inputs ...        */
+    FINCH_ERR_UNSUPPORTED = 2,         /* no sm_100 device, head_dim / dtype the kernels do not cover            */
+    FINCH_ERR_BAD_LAYOUT = 3,          /* pointer or stride not 16-byte aligned                                  */
+    FINCH_ERR_WORKSPACE_TOO_SMALL = 4, /* ws_bytes below finch_workspace_bytes                                   */
+    FINCH_ERR_OOM = 5,                 /* host or device allocation of the context failed                        */
+    FINCH_ERR_CUDA = 6,                /* a CUDA runtime/driver call failed (launch error, bad stream ...)        */
+    FINCH_ERR_DEVICE_STATUS = 7        /* finch_device_status found a non-zero status word                       */
+} finch_status;
+
+typedef enum { FINCH_F32 = 0, FINCH_BF16 = 1 } finch_dtype;
+
+typedef enum { FINCH_GROUP_PER_KV_HEAD = 0, FINCH_GROUP_PER_LAYER = 1 } finch_group_mode;
+
+/* Bits of the device status word. */
+enum {
+    FINCH_DEV_BAD_BATCH = 1,   /* device-side batch metadata exceeds the host bounds given in finch_batch      */
+    FINCH_DEV_TIMEOUT = 2,     /* a bounded wait inside a kernel ran out                                       */
+    FINCH_DEV_BAD_INDEX = 4    /* finch_compact met a kept index outside [0, N_b)                              */
+};
+
+typedef struct {
+    int32_t n_layers, n_q_heads, n_kv_heads, head_dim; /* head_dim: a multiple of 32, at most 256             */
+    int32_t dtype;       /* finch_dtype of Q, K and V                                                         */
+    int32_t group_mode;  /* finch_group_mode                                                                  */
+    float scale;         /* logit scale; 0 selects 1/sqrt(head_dim) (Background, the attention equation)      */
+    int32_t max_batch, max_prompt, max_candidates; /* upper bounds used for validation                        */
+    int32_t device;      /* CUDA device ordinal; negative = validation-only context                           */
+} finch_config;
+
+typedef struct {
+    void *ptr;
+    int64_t stride_layer, stride_head, stride_tok; /* in elements */
+} finch_tensor;
+
+typedef struct {
+    int32_t batch;
+    const int32_t *q_off, *chunk_off, *cache_off; /* device, [batch+1]                                        */
+    const int32_t *cache_len, *budget;            /* device, [batch]; budget[b] = r, at most the capacity     */
+    int32_t total_q, total_chunk, total_cache;    /* host copies of q_off[batch], chunk_off[batch], cache_off[batch] */
+    int32_t max_q, max_cache, max_chunk, max_budget; /* host upper bounds over the requests (grid sizing)      */
+} finch_batch;
+
+/* Create a context for one model shape on one device.  Fails with FINCH_ERR_UNSUPPORTED when the device is not
+ * compute capability 10.x or the shape is not covered, FINCH_ERR_INVALID_ARG on inconsistent fields
+ * (n_q_heads not a multiple of n_kv_heads, non-positive sizes).  *out is set only on success. */
+finch_status finch_ctx_create(const finch_config *cfg, finch_ctx **out);
+
+/* Free the context and its status word.  NULL is ignored.  Work still in flight must be synchronised first. */
+void finch_ctx_destroy(finch_ctx *ctx);
+
+/* Bytes of device workspace that finch_score / finch_select / finch_step need for this batch (the maximum over
+ * the three; finch_step includes room for the scores when the caller passes scores == NULL).  Pure host
+ * arithmetic: callable without touching the device. */
+finch_status finch_workspace_bytes(const finch_ctx *ctx, const finch_batch *batch, size_t *out);
+
+/* Prompt-guided scoring (Method, bullets "Sum over heads", "Extract prompt-guided submatrix", "Selection of top r
+ * position" up to A^agg; Background, the attention equation):
+ *     s[h,p,j]  = scale * <q[h,p], k[kv(h),j]>          for the candidates j < N_b
+ *     w[h,p,j]  = exp(s[h,p,j] - lse[h,p])               softmax over the candidates only
+ *     scores[j] = sum over the group's heads h and the prompt rows p of w[h,p,j]
+ * The normalisation bullet's factor count(A != 0)/(m+c) is a constant on this path (prompt rows see every
+ * candidate) and is not applied.  row_lse may be NULL (it then lives in the workspace).  Entries of `scores`
+ * beyond N_b are left untouched.  bf16 inputs with at least 64 prompt rows take the tensor-core path, everything
+ * else warp-level dot products; accumulation, softmax and the column sums are fp32 in a fixed order, so results
+ * are run-to-run identical. */
+finch_status finch_score(finch_ctx *ctx, const finch_tensor *prompt_q, const finch_tensor *cache_k,
+                         const finch_tensor *chunk_k, const finch_batch *batch, float *scores, float *row_lse,
+                         void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Top-r selection (Method, bullet "Selection of top r position": t = top-r(A^agg, r)).  For every layer, group and
+ * request keeps r' = min(budget[b], N_b) candidates with the largest scores; among equal scores the lower
+ * candidate index wins; -0 equals +0; a NaN ranks below every number.  Writes the kept candidate indices in
+ * strictly increasing order to kept_idx and r' to out_len[b].  No full sort is performed.  ws may be NULL. */
+finch_status finch_select(finch_ctx *ctx, const float *scores, const finch_batch *batch, int32_t *kept_idx,
+                          int32_t *out_len, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Cache management (Method, paragraph "Managing the Cache"; "Compression Output"): copies the K and V rows and the
+ * positions of the kept candidates, bit for bit, into rows [0, out_len[b]) of each request's region of
+ * out_k / out_v / out_pos, for every KV head of the group.  out_* must not overlap cache_* or chunk_* (the gather
+ * runs in parallel; coinciding base pointers are rejected with FINCH_ERR_INVALID_ARG).  cache_pos may be NULL only
+ * if max_cache is 0. */
+finch_status finch_compact(finch_ctx *ctx, const int32_t *kept_idx, const int32_t *out_len,
+                           const finch_tensor *cache_k, const finch_tensor *cache_v, const int32_t *cache_pos,
+                           const finch_tensor *chunk_k, const finch_tensor *chunk_v, const int32_t *chunk_pos,
+                           const finch_batch *batch, const finch_tensor *out_k, const finch_tensor *out_v,
+                           int32_t *out_pos, void *cuda_stream);
+
+/* The fused step  finch_step(prompt_q, cache_kv, chunk_kv, budget) -> cache_kv, kept_positions:
+ * score -> select -> compact enqueued back to back with no host synchronisation in between.  `scores` may be NULL
+ * (they then live in the workspace).  kept_idx receives the kept candidate indices, out_pos their original token
+ * positions.  Same argument rules as the three calls above. */
+finch_status finch_step(finch_ctx *ctx, const finch_tensor *prompt_q, const finch_tensor *cache_k,
+                        const finch_tensor *cache_v, const int32_t *cache_pos, const finch_tensor *chunk_k,
+                        const finch_tensor *chunk_v, const int32_t *chunk_pos, const finch_batch *batch,
+                        const finch_tensor *out_k, const finch_tensor *out_v, int32_t *out_pos, int32_t *kept_idx,
+                        int32_t *out_len, float *scores, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Synchronises `cuda_stream`, copies the status word to *out (host) and clears it.  Returns FINCH_ERR_DEVICE_STATUS
+ * when the word was non-zero, FINCH_ERR_CUDA when the stream reports an error. */
+finch_status finch_device_status(finch_ctx *ctx, void *cuda_stream, int32_t *out);
+
+/* Static, NUL-terminated description of a status code. */
+const char *finch_status_string(finch_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FINCH_H_ */

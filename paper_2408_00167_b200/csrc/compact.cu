@@ -1,0 +1,79 @@
+// Cache compaction: gather the kept K/V rows and positions into the next cache, in kept (ascending) order.
+//
+// One CTA copies kRowsPerCta output rows of one unit (layer, selection group, request) for every KV head of the
+// group, K and V, as 16-byte pieces: consecutive threads move consecutive pieces of a row, so both the gathered
+// reads (whole rows) and the writes (contiguous rows) are fully coalesced 128-bit accesses.
+#include "finch_internal.cuh"
+
+namespace finch {
+namespace {
+
+constexpr int kRowsPerCta = 32;
+constexpr int kCompactThreads = 256;
+
+__global__ void __launch_bounds__(kCompactThreads)
+compact_kernel(ModelView mv, BatchView bv, const int *kept_idx, const int *out_len, TensorView cache_k,
+               TensorView cache_v, const int *cache_pos, TensorView chunk_k, TensorView chunk_v, const int *chunk_pos,
+               TensorView out_k, TensorView out_v, int *out_pos, int *status) {
+    __shared__ int src_idx[kRowsPerCta];
+    const UnitInfo u = unit_info(mv, bv, blockIdx.y, blockIdx.z);
+    if (!u.ok) {
+        if (threadIdx.x == 0) atomicOr(status, FINCH_DEV_BAD_BATCH);
+        return;
+    }
+    int r = out_len[u.b];
+    if (r > u.cap) r = u.cap;
+    const int i0 = blockIdx.x * kRowsPerCta;
+    if (i0 >= r) return;
+    const int rows = min(kRowsPerCta, r - i0);
+    const int64_t unit_off = ((int64_t)u.l * mv.G + u.G) * bv.total_cache + u.cache0;
+
+    if (threadIdx.x < rows) {
+        int j = kept_idx[unit_off + i0 + threadIdx.x];
+        if (j < 0 || j >= u.N) {
+            atomicOr(status, FINCH_DEV_BAD_INDEX);
+            j = -1;
+        } else {
+            out_pos[unit_off + i0 + threadIdx.x] = j < u.c ? cache_pos[unit_off + j] : chunk_pos[u.chunk0 + j - u.c];
+        }
+        src_idx[threadIdx.x] = j;
+    }
+    __syncthreads();
+
+    const int pieces = mv.d * mv.elem_bytes / 16;  // 16-byte pieces per row
+    const int per_row = pieces * 2 * mv.kvpg;      // K and V, every KV head of the group
+    for (int e = threadIdx.x; e < rows * per_row; e += kCompactThreads) {
+        const int row = e / per_row, rem = e % per_row;
+        const int piece = rem % pieces, which = rem / pieces;  // which = kv * 2 + {0: K, 1: V}
+        const int kvh = u.G * mv.kvpg + which / 2;
+        const bool is_v = which & 1;
+        const int j = src_idx[row];
+        if (j < 0) continue;
+        const TensorView &src = j < u.c ? (is_v ? cache_v : cache_k) : (is_v ? chunk_v : chunk_k);
+        const int64_t src_tok = j < u.c ? u.cache0 + j : u.chunk0 + j - u.c;
+        const TensorView &dst = is_v ? out_v : out_k;
+        const int64_t se = (int64_t)u.l * src.stride_layer + (int64_t)kvh * src.stride_head + src_tok * src.stride_tok;
+        const int64_t de = (int64_t)u.l * dst.stride_layer + (int64_t)kvh * dst.stride_head +
+                           (int64_t)(u.cache0 + i0 + row) * dst.stride_tok;
+        const uint4 v = __ldg((const uint4 *)(src.ptr + se * mv.elem_bytes) + piece);
+        ((uint4 *)(const_cast<char *>(dst.ptr) + de * mv.elem_bytes))[piece] = v;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_compact(const Ctx &ctx, const int *kept_idx, const int *out_len, const TensorView &cache_k,
+                           const TensorView &cache_v, const int *cache_pos, const TensorView &chunk_k,
+                           const TensorView &chunk_v, const int *chunk_pos, const BatchView &bv, const TensorView &out_k,
+                           const TensorView &out_v, int *out_pos, cudaStream_t stream) {
+    const ModelView &mv = ctx.model;
+    const int units = mv.L * mv.G;
+    const int row_blocks = (bv.max_budget + kRowsPerCta - 1) / kRowsPerCta;
+    if (units == 0 || bv.batch == 0 || row_blocks == 0) return cudaSuccess;
+    dim3 grid(row_blocks, units, bv.batch);
+    compact_kernel<<<grid, kCompactThreads, 0, stream>>>(mv, bv, kept_idx, out_len, cache_k, cache_v, cache_pos, chunk_k,
+                                                         chunk_v, chunk_pos, out_k, out_v, out_pos, ctx.d_status);
+    return cudaGetLastError();
+}
+
+}  // namespace finch

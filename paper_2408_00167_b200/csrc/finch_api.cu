@@ -1,0 +1,278 @@
+// Host side of the C ABI: context, argument validation, workspace layout and kernel dispatch.
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "finch_internal.cuh"
+
+using namespace finch;
+
+struct finch_ctx : public Ctx {};
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+inline bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
+
+finch_status check_tensor(const finch_ctx *ctx, const finch_tensor *t, bool allow_null_ptr) {
+    if (!t) return FINCH_ERR_INVALID_ARG;
+    if (!t->ptr) return allow_null_ptr ? FINCH_OK : FINCH_ERR_INVALID_ARG;
+    const int64_t e = ctx->model.elem_bytes;
+    if (!aligned16(t->ptr) || (t->stride_layer * e) % 16 || (t->stride_head * e) % 16 || (t->stride_tok * e) % 16)
+        return FINCH_ERR_BAD_LAYOUT;
+    if (t->stride_tok < ctx->model.d || t->stride_head < 0 || t->stride_layer < 0) return FINCH_ERR_INVALID_ARG;
+    return FINCH_OK;
+}
+
+finch_status check_batch(const finch_ctx *ctx, const finch_batch *b) {
+    if (!ctx || !b) return FINCH_ERR_INVALID_ARG;
+    if (b->batch < 0 || b->batch > ctx->cfg.max_batch) return FINCH_ERR_INVALID_ARG;
+    if (b->total_q < 0 || b->total_chunk < 0 || b->total_cache < 0) return FINCH_ERR_INVALID_ARG;
+    if (b->max_q < 0 || b->max_cache < 0 || b->max_chunk < 0 || b->max_budget < 0) return FINCH_ERR_INVALID_ARG;
+    if (b->max_q > ctx->cfg.max_prompt) return FINCH_ERR_INVALID_ARG;
+    if ((int64_t)b->max_cache + b->max_chunk > ctx->cfg.max_candidates) return FINCH_ERR_INVALID_ARG;
+    if (b->max_q > b->total_q || b->max_chunk > b->total_chunk || b->max_cache > b->total_cache ||
+        b->max_budget > b->total_cache)
+        return FINCH_ERR_INVALID_ARG;
+    if (b->batch > 0 && (!b->q_off || !b->chunk_off || !b->cache_off || !b->cache_len || !b->budget))
+        return FINCH_ERR_INVALID_ARG;
+    return FINCH_OK;
+}
+
+struct WsLayout {
+    size_t lse_off, lse_bytes;        // row log-sum-exp when the caller gives none
+    size_t scores_off, scores_bytes;  // scores inside finch_step when the caller gives none
+    size_t total;
+};
+
+WsLayout ws_layout(const finch_ctx *ctx, const finch_batch *b) {
+    WsLayout w{};
+    const ModelView &mv = ctx->model;
+    w.lse_off = 0;
+    w.lse_bytes = align_up((size_t)mv.L * mv.Hq * (size_t)b->total_q * sizeof(float));
+    w.scores_off = w.lse_off + w.lse_bytes;
+    w.scores_bytes = align_up((size_t)mv.L * mv.G * ((size_t)b->total_cache + b->total_chunk) * sizeof(float));
+    w.total = w.scores_off + w.scores_bytes;
+    if (w.total == 0) w.total = kAlign;
+    return w;
+}
+
+finch_status cuda_status(cudaError_t e) { return e == cudaSuccess ? FINCH_OK : FINCH_ERR_CUDA; }
+
+bool same_base(const finch_tensor *a, const finch_tensor *b) { return a && b && a->ptr && a->ptr == b->ptr; }
+
+finch_status validate_score(const finch_ctx *ctx, const finch_tensor *q, const finch_tensor *cache_k,
+                            const finch_tensor *chunk_k, const finch_batch *batch) {
+    finch_status s = check_batch(ctx, batch);
+    if (s) return s;
+    if ((s = check_tensor(ctx, q, batch->total_q == 0))) return s;
+    if ((s = check_tensor(ctx, cache_k, batch->total_cache == 0))) return s;
+    if ((s = check_tensor(ctx, chunk_k, batch->total_chunk == 0))) return s;
+    if (batch->max_q == 0 && batch->batch > 0) return FINCH_ERR_INVALID_ARG;  // scoring needs prompt rows
+    return FINCH_OK;
+}
+
+finch_status validate_compact(const finch_ctx *ctx, const int32_t *kept_idx, const int32_t *out_len,
+                              const finch_tensor *cache_k, const finch_tensor *cache_v, const int32_t *cache_pos,
+                              const finch_tensor *chunk_k, const finch_tensor *chunk_v, const int32_t *chunk_pos,
+                              const finch_batch *batch, const finch_tensor *out_k, const finch_tensor *out_v,
+                              const int32_t *out_pos) {
+    finch_status s = check_batch(ctx, batch);
+    if (s) return s;
+    const bool no_cache = batch->total_cache == 0, no_chunk = batch->total_chunk == 0;
+    if ((s = check_tensor(ctx, cache_k, no_cache))) return s;
+    if ((s = check_tensor(ctx, cache_v, no_cache))) return s;
+    if ((s = check_tensor(ctx, chunk_k, no_chunk))) return s;
+    if ((s = check_tensor(ctx, chunk_v, no_chunk))) return s;
+    if ((s = check_tensor(ctx, out_k, no_cache))) return s;
+    if ((s = check_tensor(ctx, out_v, no_cache))) return s;
+    if (!no_cache && (!out_pos || !kept_idx)) return FINCH_ERR_INVALID_ARG;
+    if (!no_chunk && !chunk_pos) return FINCH_ERR_INVALID_ARG;
+    if (batch->max_cache > 0 && !cache_pos) return FINCH_ERR_INVALID_ARG;
+    if (batch->batch > 0 && !out_len) return FINCH_ERR_INVALID_ARG;
+    const finch_tensor *outs[2] = {out_k, out_v};
+    const finch_tensor *ins[4] = {cache_k, cache_v, chunk_k, chunk_v};
+    for (auto o : outs)
+        for (auto i : ins)
+            if (same_base(o, i)) return FINCH_ERR_INVALID_ARG;
+    if (same_base(out_k, out_v)) return FINCH_ERR_INVALID_ARG;
+    return FINCH_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *finch_status_string(finch_status s) {
+    switch (s) {
+        case FINCH_OK: return "ok";
+        case FINCH_ERR_INVALID_ARG: return "invalid argument";
+        case FINCH_ERR_UNSUPPORTED: return "unsupported device or shape";
+        case FINCH_ERR_BAD_LAYOUT: return "pointer or stride not 16-byte aligned";
+        case FINCH_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case FINCH_ERR_OOM: return "out of memory";
+        case FINCH_ERR_CUDA: return "CUDA error";
+        case FINCH_ERR_DEVICE_STATUS: return "device status word is non-zero";
+    }
+    return "unknown status";
+}
+
+finch_status finch_ctx_create(const finch_config *cfg, finch_ctx **out) {
+    if (!cfg || !out) return FINCH_ERR_INVALID_ARG;
+    if (cfg->n_layers <= 0 || cfg->n_q_heads <= 0 || cfg->n_kv_heads <= 0 || cfg->head_dim <= 0)
+        return FINCH_ERR_INVALID_ARG;
+    if (cfg->n_q_heads % cfg->n_kv_heads) return FINCH_ERR_INVALID_ARG;
+    if (cfg->dtype != FINCH_F32 && cfg->dtype != FINCH_BF16) return FINCH_ERR_INVALID_ARG;
+    if (cfg->group_mode != FINCH_GROUP_PER_KV_HEAD && cfg->group_mode != FINCH_GROUP_PER_LAYER)
+        return FINCH_ERR_INVALID_ARG;
+    if (cfg->max_batch <= 0 || cfg->max_prompt <= 0 || cfg->max_candidates <= 0) return FINCH_ERR_INVALID_ARG;
+    if (!(cfg->scale >= 0.f) || isinf(cfg->scale)) return FINCH_ERR_INVALID_ARG;
+    if (cfg->head_dim % 32 || cfg->head_dim > 256) return FINCH_ERR_UNSUPPORTED;
+    if ((int64_t)cfg->n_layers * cfg->n_kv_heads > 65535 || cfg->max_batch > 65535) return FINCH_ERR_UNSUPPORTED;
+
+    finch_ctx *ctx = new (std::nothrow) finch_ctx();
+    if (!ctx) return FINCH_ERR_OOM;
+    ctx->cfg = *cfg;
+    ModelView &mv = ctx->model;
+    mv.L = cfg->n_layers;
+    mv.Hq = cfg->n_q_heads;
+    mv.Hkv = cfg->n_kv_heads;
+    mv.d = cfg->head_dim;
+    mv.G = cfg->group_mode == FINCH_GROUP_PER_KV_HEAD ? cfg->n_kv_heads : 1;
+    mv.hpg = mv.Hq / mv.G;
+    mv.g = mv.Hq / mv.Hkv;
+    mv.kvpg = mv.Hkv / mv.G;
+    mv.scale = cfg->scale > 0.f ? cfg->scale : 1.0f / sqrtf((float)cfg->head_dim);
+    mv.elem_bytes = cfg->dtype == FINCH_F32 ? 4 : 2;
+    ctx->d_status = nullptr;
+    ctx->dry = cfg->device < 0;
+    ctx->sm_count = 0;
+    if (!ctx->dry) {
+        int n_dev = 0;
+        cudaDeviceProp prop;
+        if (cudaGetDeviceCount(&n_dev) != cudaSuccess || cfg->device >= n_dev ||
+            cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess || prop.major != 10) {
+            (void)cudaGetLastError();
+            delete ctx;
+            return FINCH_ERR_UNSUPPORTED;
+        }
+        ctx->sm_count = prop.multiProcessorCount;
+        if (cudaSetDevice(cfg->device) != cudaSuccess || cudaMalloc(&ctx->d_status, sizeof(int)) != cudaSuccess) {
+            (void)cudaGetLastError();
+            delete ctx;
+            return FINCH_ERR_OOM;
+        }
+        if (cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess) {
+            cudaFree(ctx->d_status);
+            delete ctx;
+            return FINCH_ERR_CUDA;
+        }
+    }
+    *out = ctx;
+    return FINCH_OK;
+}
+
+void finch_ctx_destroy(finch_ctx *ctx) {
+    if (!ctx) return;
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    delete ctx;
+}
+
+finch_status finch_workspace_bytes(const finch_ctx *ctx, const finch_batch *batch, size_t *out) {
+    if (!out) return FINCH_ERR_INVALID_ARG;
+    finch_status s = check_batch(ctx, batch);
+    if (s) return s;
+    *out = ws_layout(ctx, batch).total;
+    return FINCH_OK;
+}
+
+finch_status finch_score(finch_ctx *ctx, const finch_tensor *prompt_q, const finch_tensor *cache_k,
+                         const finch_tensor *chunk_k, const finch_batch *batch, float *scores, float *row_lse, void *ws,
+                         size_t ws_bytes, void *cuda_stream) {
+    finch_status s = validate_score(ctx, prompt_q, cache_k, chunk_k, batch);
+    if (s) return s;
+    const WsLayout w = ws_layout(ctx, batch);
+    if (!scores && (size_t)batch->total_cache + batch->total_chunk > 0) return FINCH_ERR_INVALID_ARG;
+    if (!row_lse) {
+        if (!ws) return FINCH_ERR_INVALID_ARG;
+        if (!aligned16(ws)) return FINCH_ERR_BAD_LAYOUT;
+        if (ws_bytes < w.lse_off + w.lse_bytes) return FINCH_ERR_WORKSPACE_TOO_SMALL;
+        row_lse = (float *)((char *)ws + w.lse_off);
+    }
+    if (ctx->dry) return FINCH_ERR_UNSUPPORTED;
+    return cuda_status(launch_score_simt(*ctx, view_of(prompt_q), view_of(cache_k), view_of(chunk_k), view_of(batch),
+                                         scores, row_lse, (cudaStream_t)cuda_stream));
+}
+
+finch_status finch_select(finch_ctx *ctx, const float *scores, const finch_batch *batch, int32_t *kept_idx,
+                          int32_t *out_len, void *ws, size_t ws_bytes, void *cuda_stream) {
+    (void)ws;
+    (void)ws_bytes;
+    finch_status s = check_batch(ctx, batch);
+    if (s) return s;
+    if (batch->batch > 0 && !out_len) return FINCH_ERR_INVALID_ARG;
+    if ((size_t)batch->total_cache + batch->total_chunk > 0 && !scores) return FINCH_ERR_INVALID_ARG;
+    if (batch->total_cache > 0 && !kept_idx) return FINCH_ERR_INVALID_ARG;
+    if (ctx->dry) return FINCH_ERR_UNSUPPORTED;
+    return cuda_status(launch_select(*ctx, scores, view_of(batch), kept_idx, out_len, (cudaStream_t)cuda_stream));
+}
+
+finch_status finch_compact(finch_ctx *ctx, const int32_t *kept_idx, const int32_t *out_len, const finch_tensor *cache_k,
+                           const finch_tensor *cache_v, const int32_t *cache_pos, const finch_tensor *chunk_k,
+                           const finch_tensor *chunk_v, const int32_t *chunk_pos, const finch_batch *batch,
+                           const finch_tensor *out_k, const finch_tensor *out_v, int32_t *out_pos, void *cuda_stream) {
+    finch_status s = validate_compact(ctx, kept_idx, out_len, cache_k, cache_v, cache_pos, chunk_k, chunk_v, chunk_pos,
+                                      batch, out_k, out_v, out_pos);
+    if (s) return s;
+    if (ctx->dry) return FINCH_ERR_UNSUPPORTED;
+    return cuda_status(launch_compact(*ctx, kept_idx, out_len, view_of(cache_k), view_of(cache_v), cache_pos,
+                                      view_of(chunk_k), view_of(chunk_v), chunk_pos, view_of(batch), view_of(out_k),
+                                      view_of(out_v), out_pos, (cudaStream_t)cuda_stream));
+}
+
+finch_status finch_step(finch_ctx *ctx, const finch_tensor *prompt_q, const finch_tensor *cache_k,
+                        const finch_tensor *cache_v, const int32_t *cache_pos, const finch_tensor *chunk_k,
+                        const finch_tensor *chunk_v, const int32_t *chunk_pos, const finch_batch *batch,
+                        const finch_tensor *out_k, const finch_tensor *out_v, int32_t *out_pos, int32_t *kept_idx,
+                        int32_t *out_len, float *scores, void *ws, size_t ws_bytes, void *cuda_stream) {
+    finch_status s = validate_score(ctx, prompt_q, cache_k, chunk_k, batch);
+    if (s) return s;
+    if ((s = validate_compact(ctx, kept_idx, out_len, cache_k, cache_v, cache_pos, chunk_k, chunk_v, chunk_pos, batch,
+                              out_k, out_v, out_pos)))
+        return s;
+    if (!ws) return FINCH_ERR_INVALID_ARG;
+    if (!aligned16(ws)) return FINCH_ERR_BAD_LAYOUT;
+    const WsLayout w = ws_layout(ctx, batch);
+    if (ws_bytes < (scores ? w.lse_off + w.lse_bytes : w.total)) return FINCH_ERR_WORKSPACE_TOO_SMALL;
+    float *row_lse = (float *)((char *)ws + w.lse_off);
+    if (!scores) scores = (float *)((char *)ws + w.scores_off);
+    if (ctx->dry) return FINCH_ERR_UNSUPPORTED;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const BatchView bv = view_of(batch);
+    cudaError_t e = launch_score_simt(*ctx, view_of(prompt_q), view_of(cache_k), view_of(chunk_k), bv, scores, row_lse,
+                                      stream);
+    if (e == cudaSuccess) e = launch_select(*ctx, scores, bv, kept_idx, out_len, stream);
+    if (e == cudaSuccess)
+        e = launch_compact(*ctx, kept_idx, out_len, view_of(cache_k), view_of(cache_v), cache_pos, view_of(chunk_k),
+                           view_of(chunk_v), chunk_pos, bv, view_of(out_k), view_of(out_v), out_pos, stream);
+    return cuda_status(e);
+}
+
+finch_status finch_device_status(finch_ctx *ctx, void *cuda_stream, int32_t *out) {
+    if (!ctx || !out) return FINCH_ERR_INVALID_ARG;
+    if (ctx->dry) return FINCH_ERR_UNSUPPORTED;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    int host = 0;
+    if (cudaMemcpyAsync(&host, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaMemsetAsync(ctx->d_status, 0, sizeof(int), stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return FINCH_ERR_CUDA;
+    }
+    *out = host;
+    return host ? FINCH_ERR_DEVICE_STATUS : FINCH_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,94 @@
+// Internal declarations shared by the translation units of libfinch (not part of the public ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "finch.h"
+
+namespace finch {
+
+// Device-side view of a finch_tensor (strides in elements, head_dim contiguous).
+struct TensorView {
+    const char *ptr;
+    int64_t stride_layer, stride_head, stride_tok;
+};
+
+struct BatchView {
+    int batch;
+    const int *q_off, *chunk_off, *cache_off, *cache_len, *budget;
+    int total_q, total_chunk, total_cache;
+    int max_q, max_cache, max_chunk, max_budget;
+};
+
+struct ModelView {
+    int L, Hq, Hkv, d;
+    int G;           // selection groups per layer
+    int hpg;         // query heads per selection group
+    int g;           // query heads per KV head
+    int kvpg;        // KV heads per selection group
+    float scale;     // logit scale (natural units)
+    int elem_bytes;  // 2 (bf16) or 4 (f32)
+};
+
+struct Ctx {
+    finch_config cfg;
+    ModelView model;
+    int *d_status;  // device status word (nullptr for a validation-only context)
+    bool dry;       // validation-only context: nothing is ever enqueued
+    int sm_count;
+};
+
+inline TensorView view_of(const finch_tensor *t) {
+    return TensorView{(const char *)t->ptr, t->stride_layer, t->stride_head, t->stride_tok};
+}
+inline BatchView view_of(const finch_batch *b) {
+    return BatchView{b->batch,       b->q_off,       b->chunk_off, b->cache_off, b->cache_len, b->budget,    b->total_q,
+                     b->total_chunk, b->total_cache, b->max_q,     b->max_cache, b->max_chunk, b->max_budget};
+}
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// What every kernel needs to know about one unit = (layer, selection group, request).
+struct UnitInfo {
+    int l, G, b;
+    int n_q, c, m, N;
+    int q0, cache0, chunk0, cap;
+    bool ok;
+};
+
+__device__ __forceinline__ UnitInfo unit_info(const ModelView &mv, const BatchView &bv, int unit, int b) {
+    UnitInfo u;
+    u.l = unit / mv.G;
+    u.G = unit % mv.G;
+    u.b = b;
+    u.q0 = bv.q_off[b];
+    u.n_q = bv.q_off[b + 1] - u.q0;
+    u.cache0 = bv.cache_off[b];
+    u.cap = bv.cache_off[b + 1] - u.cache0;
+    u.chunk0 = bv.chunk_off[b];
+    u.c = bv.cache_len[b];
+    u.m = bv.chunk_off[b + 1] - u.chunk0;
+    u.N = u.c + u.m;
+    u.ok = u.n_q >= 0 && u.n_q <= bv.max_q && u.c >= 0 && u.c <= bv.max_cache && u.m >= 0 && u.m <= bv.max_chunk &&
+           u.c <= u.cap;
+    return u;
+}
+
+// ---- launchers implemented in the kernel files; each returns the cudaError_t of its launches ----
+
+// warp-level dot-product scoring (any dtype, any prompt length)
+cudaError_t launch_score_simt(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
+                              const BatchView &bv, float *scores, float *row_lse, cudaStream_t stream);
+
+cudaError_t launch_select(const Ctx &ctx, const float *scores, const BatchView &bv, int *kept_idx, int *out_len,
+                          cudaStream_t stream);
+
+cudaError_t launch_compact(const Ctx &ctx, const int *kept_idx, const int *out_len, const TensorView &cache_k,
+                           const TensorView &cache_v, const int *cache_pos, const TensorView &chunk_k,
+                           const TensorView &chunk_v, const int *chunk_pos, const BatchView &bv, const TensorView &out_k,
+                           const TensorView &out_v, int *out_pos, cudaStream_t stream);
+
+}  // namespace finch

@@ -1,0 +1,162 @@
+// Top-r selection per (layer, selection group, request) without a sort.
+//
+// One CTA per unit.  Scores are mapped to order-preserving 32-bit keys; four 8-bit radix passes (most significant
+// digit first) locate the key T of the r-th largest score and how many candidates are strictly above it.  A final
+// ordered sweep keeps every candidate above T plus the lowest-indexed candidates equal to T until r are kept, and
+// writes the kept indices in increasing order (block-wide prefix sums over ballots).
+#include "finch_internal.cuh"
+
+namespace finch {
+namespace {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSelWarps = kSelThreads / 32;
+
+// Order-preserving key: larger score <=> larger key.  -0 is folded into +0; NaN gets key 0, below every number.
+__device__ __forceinline__ uint32_t order_key(float s) {
+    if (s != s) return 0u;
+    uint32_t u = __float_as_uint(s);
+    if ((u << 1) == 0u) u = 0u;  // -0 -> +0
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__global__ void __launch_bounds__(kSelThreads)
+select_kernel(ModelView mv, BatchView bv, const float *scores, int *kept_idx, int *out_len, int smem_keys, int *status) {
+    extern __shared__ uint32_t key_cache[];  // the first min(N, smem_keys) keys
+    __shared__ int hist[256];
+    __shared__ int warp_tot[2][kSelWarps];
+    __shared__ int sel_digit, sel_above;
+
+    const int unit = blockIdx.x;
+    const UnitInfo u = unit_info(mv, bv, unit, blockIdx.y);
+    const int N = u.N;
+    int r = bv.budget[u.b];
+    r = r < N ? r : N;
+    r = r < 0 ? 0 : r;
+    if (!u.ok || r > u.cap || r > bv.max_budget) {  // block-uniform
+        if (threadIdx.x == 0) {
+            atomicOr(status, FINCH_DEV_BAD_BATCH);
+            if (unit == 0) out_len[u.b] = 0;
+        }
+        return;
+    }
+    if (unit == 0 && threadIdx.x == 0) out_len[u.b] = r;
+    if (r == 0) return;
+
+    const float *sc = scores + ((int64_t)u.l * mv.G + u.G) * ((int64_t)bv.total_cache + bv.total_chunk) + u.cache0 +
+                      u.chunk0;
+    int *kept = kept_idx + ((int64_t)u.l * mv.G + u.G) * bv.total_cache + u.cache0;
+
+    if (r == N) {  // a budget at or above the candidate count keeps everything, in order
+        for (int j = threadIdx.x; j < N; j += kSelThreads) kept[j] = j;
+        return;
+    }
+
+    const int n_cached = N < smem_keys ? N : smem_keys;
+    for (int j = threadIdx.x; j < n_cached; j += kSelThreads) key_cache[j] = order_key(sc[j]);
+    __syncthreads();
+    auto key_at = [&](int j) -> uint32_t { return j < n_cached ? key_cache[j] : order_key(sc[j]); };
+
+    // ---- radix search for the r-th largest key
+    uint32_t prefix = 0, mask = 0;
+    int remaining = r;  // rank, among the keys matching the prefix, of the key we look for (1 = largest)
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+        __syncthreads();
+        for (int j = threadIdx.x; j < N; j += kSelThreads) {
+            const uint32_t k = key_at(j);
+            if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1);
+        }
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            // lane i owns digits 255-8i .. 248-8i (descending); find the digit where the running count reaches
+            // `remaining`
+            const int lane = threadIdx.x;
+            int mine = 0;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) mine += hist[255 - 8 * lane - t];
+            int incl = mine;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += v;
+            }
+            int above = incl - mine;
+            if (above < remaining && remaining <= incl) {
+                for (int t = 0; t < 8; ++t) {
+                    const int digit = 255 - 8 * lane - t;
+                    const int cnt = hist[digit];
+                    if (remaining <= above + cnt) {
+                        sel_digit = digit;
+                        sel_above = above;
+                        break;
+                    }
+                    above += cnt;
+                }
+            }
+        }
+        __syncthreads();
+        prefix |= (uint32_t)sel_digit << shift;
+        mask |= 255u << shift;
+        remaining -= sel_above;
+        __syncthreads();
+    }
+    const uint32_t T = prefix;
+    const int ties_to_keep = remaining;  // >= 1
+
+    // ---- ordered sweep: keep key > T, and the first `ties_to_keep` keys == T
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int base_eq = 0, base_keep = 0;
+    for (int j0 = 0; j0 < N; j0 += kSelThreads) {
+        const int j = j0 + threadIdx.x;
+        const uint32_t k = j < N ? key_at(j) : 0u;
+        const bool gt = j < N && k > T;
+        const bool eq = j < N && k == T;
+        const uint32_t eq_ballot = __ballot_sync(0xffffffffu, eq);
+        if (lane == 0) warp_tot[0][warp] = __popc(eq_ballot);
+        __syncthreads();
+        int eq_before = base_eq, eq_all = 0;
+        for (int w = 0; w < kSelWarps; ++w) {
+            const int t = warp_tot[0][w];
+            if (w < warp) eq_before += t;
+            eq_all += t;
+        }
+        eq_before += __popc(eq_ballot & ((1u << lane) - 1u));
+        const bool keep = gt || (eq && eq_before < ties_to_keep);
+        const uint32_t keep_ballot = __ballot_sync(0xffffffffu, keep);
+        if (lane == 0) warp_tot[1][warp] = __popc(keep_ballot);
+        __syncthreads();
+        int keep_before = base_keep, keep_all = 0;
+        for (int w = 0; w < kSelWarps; ++w) {
+            const int t = warp_tot[1][w];
+            if (w < warp) keep_before += t;
+            keep_all += t;
+        }
+        keep_before += __popc(keep_ballot & ((1u << lane) - 1u));
+        if (keep) kept[keep_before] = j;
+        base_eq += eq_all;
+        base_keep += keep_all;
+        // no barrier needed here: warp_tot[0] was last read before the second barrier above, and warp_tot[1] is
+        // rewritten only after the next iteration's first barrier
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_select(const Ctx &ctx, const float *scores, const BatchView &bv, int *kept_idx, int *out_len,
+                          cudaStream_t stream) {
+    const ModelView &mv = ctx.model;
+    const int units = mv.L * mv.G;
+    if (units == 0 || bv.batch == 0) return cudaSuccess;
+    const int max_n = bv.max_cache + bv.max_chunk;
+    int smem_keys = max_n < 40960 ? max_n : 40960;  // up to 160 KiB of keys on chip; longer inputs re-read global
+    if (smem_keys < 1) smem_keys = 1;
+    const size_t smem = (size_t)smem_keys * sizeof(uint32_t);
+    cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    dim3 grid(units, bv.batch);
+    select_kernel<<<grid, kSelThreads, smem, stream>>>(mv, bv, scores, kept_idx, out_len, smem_keys, ctx.d_status);
+    return cudaGetLastError();
+}
+
+}  // namespace finch
