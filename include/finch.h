@@ -129,7 +129,7 @@ finch_status finch_workspace_bytes(const finch_ctx *ctx, const finch_batch *batc
  *     w[h,p,j]  = exp(s[h,p,j] - lse[h,p])               softmax over the candidates only
  *     scores[j] = sum over the group's heads h and the prompt rows p of w[h,p,j]
  * The normalisation bullet's factor count(A != 0)/(m+c) is a constant on this path (prompt rows see every
- * candidate) and is not applied.  row_lse may be NULL (it then lives in the workspace).  Entries of `scores`
+ * candidate) and is not applied.  row_lse may be NULL; the workspace is always required.  Entries of `scores`
  * beyond N_b are left untouched.  bf16 inputs with at least 64 prompt rows take the tensor-core path, everything
  * else warp-level dot products; accumulation, softmax and the column sums are fp32 in a fixed order, so results
  * are run-to-run identical. */
@@ -168,6 +168,10 @@ finch_status finch_step(finch_ctx *ctx, const finch_tensor *prompt_q, const finc
 /* Synchronises `cuda_stream`, copies the status word to *out (host) and clears it.  Returns FINCH_ERR_DEVICE_STATUS
  * when the word was non-zero, FINCH_ERR_CUDA when the stream reports an error. */
 finch_status finch_device_status(finch_ctx *ctx, void *cuda_stream, int32_t *out);
+
+/* Number of CUDA kernels this context has enqueued since it was created (host counter, for instrumentation).
+ * The paper has no counterpart. */
+finch_status finch_launch_count(const finch_ctx *ctx, uint64_t *out);
 
 /* Static, NUL-terminated description of a status code. */
 const char *finch_status_string(finch_status s);

@@ -73,6 +73,7 @@ cudaError_t launch_compact(const Ctx &ctx, const int *kept_idx, const int *out_l
     dim3 grid(row_blocks, units, bv.batch);
     compact_kernel<<<grid, kCompactThreads, 0, stream>>>(mv, bv, kept_idx, out_len, cache_k, cache_v, cache_pos, chunk_k,
                                                          chunk_v, chunk_pos, out_k, out_v, out_pos, ctx.d_status);
+    ctx.launches += 1;
     return cudaGetLastError();
 }
 

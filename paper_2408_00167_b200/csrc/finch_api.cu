@@ -42,7 +42,7 @@ finch_status check_batch(const finch_ctx *ctx, const finch_batch *b) {
 }
 
 struct WsLayout {
-    size_t lse_off, lse_bytes;        // row log-sum-exp when the caller gives none
+    size_t lse_off, lse_bytes;        // per prompt row (max, 1/sum) of the softmax, float2
     size_t scores_off, scores_bytes;  // scores inside finch_step when the caller gives none
     size_t total;
 };
@@ -51,7 +51,7 @@ WsLayout ws_layout(const finch_ctx *ctx, const finch_batch *b) {
     WsLayout w{};
     const ModelView &mv = ctx->model;
     w.lse_off = 0;
-    w.lse_bytes = align_up((size_t)mv.L * mv.Hq * (size_t)b->total_q * sizeof(float));
+    w.lse_bytes = align_up((size_t)mv.L * mv.Hq * (size_t)b->total_q * sizeof(float2));
     w.scores_off = w.lse_off + w.lse_bytes;
     w.scores_bytes = align_up((size_t)mv.L * mv.G * ((size_t)b->total_cache + b->total_chunk) * sizeof(float));
     w.total = w.scores_off + w.scores_bytes;
@@ -149,6 +149,7 @@ finch_status finch_ctx_create(const finch_config *cfg, finch_ctx **out) {
     ctx->d_status = nullptr;
     ctx->dry = cfg->device < 0;
     ctx->sm_count = 0;
+    ctx->launches = 0;
     if (!ctx->dry) {
         int n_dev = 0;
         cudaDeviceProp prop;
@@ -195,15 +196,13 @@ finch_status finch_score(finch_ctx *ctx, const finch_tensor *prompt_q, const fin
     if (s) return s;
     const WsLayout w = ws_layout(ctx, batch);
     if (!scores && (size_t)batch->total_cache + batch->total_chunk > 0) return FINCH_ERR_INVALID_ARG;
-    if (!row_lse) {
-        if (!ws) return FINCH_ERR_INVALID_ARG;
-        if (!aligned16(ws)) return FINCH_ERR_BAD_LAYOUT;
-        if (ws_bytes < w.lse_off + w.lse_bytes) return FINCH_ERR_WORKSPACE_TOO_SMALL;
-        row_lse = (float *)((char *)ws + w.lse_off);
-    }
+    if (!ws) return FINCH_ERR_INVALID_ARG;
+    if (!aligned16(ws)) return FINCH_ERR_BAD_LAYOUT;
+    if (ws_bytes < w.lse_off + w.lse_bytes) return FINCH_ERR_WORKSPACE_TOO_SMALL;
+    float2 *row_stats = (float2 *)((char *)ws + w.lse_off);
     if (ctx->dry) return FINCH_ERR_UNSUPPORTED;
     return cuda_status(launch_score_simt(*ctx, view_of(prompt_q), view_of(cache_k), view_of(chunk_k), view_of(batch),
-                                         scores, row_lse, (cudaStream_t)cuda_stream));
+                                         scores, row_stats, row_lse, (cudaStream_t)cuda_stream));
 }
 
 finch_status finch_select(finch_ctx *ctx, const float *scores, const finch_batch *batch, int32_t *kept_idx,
@@ -246,18 +245,24 @@ finch_status finch_step(finch_ctx *ctx, const finch_tensor *prompt_q, const finc
     if (!aligned16(ws)) return FINCH_ERR_BAD_LAYOUT;
     const WsLayout w = ws_layout(ctx, batch);
     if (ws_bytes < (scores ? w.lse_off + w.lse_bytes : w.total)) return FINCH_ERR_WORKSPACE_TOO_SMALL;
-    float *row_lse = (float *)((char *)ws + w.lse_off);
+    float2 *row_stats = (float2 *)((char *)ws + w.lse_off);
     if (!scores) scores = (float *)((char *)ws + w.scores_off);
     if (ctx->dry) return FINCH_ERR_UNSUPPORTED;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     const BatchView bv = view_of(batch);
-    cudaError_t e = launch_score_simt(*ctx, view_of(prompt_q), view_of(cache_k), view_of(chunk_k), bv, scores, row_lse,
-                                      stream);
+    cudaError_t e = launch_score_simt(*ctx, view_of(prompt_q), view_of(cache_k), view_of(chunk_k), bv, scores, row_stats,
+                                      nullptr, stream);
     if (e == cudaSuccess) e = launch_select(*ctx, scores, bv, kept_idx, out_len, stream);
     if (e == cudaSuccess)
         e = launch_compact(*ctx, kept_idx, out_len, view_of(cache_k), view_of(cache_v), cache_pos, view_of(chunk_k),
                            view_of(chunk_v), chunk_pos, bv, view_of(out_k), view_of(out_v), out_pos, stream);
     return cuda_status(e);
+}
+
+finch_status finch_launch_count(const finch_ctx *ctx, uint64_t *out) {
+    if (!ctx || !out) return FINCH_ERR_INVALID_ARG;
+    *out = ctx->launches;
+    return FINCH_OK;
 }
 
 finch_status finch_device_status(finch_ctx *ctx, void *cuda_stream, int32_t *out) {

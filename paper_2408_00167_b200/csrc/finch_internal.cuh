@@ -38,6 +38,7 @@ struct Ctx {
     int *d_status;  // device status word (nullptr for a validation-only context)
     bool dry;       // validation-only context: nothing is ever enqueued
     int sm_count;
+    mutable uint64_t launches;  // kernels enqueued through this context
 };
 
 inline TensorView view_of(const finch_tensor *t) {
@@ -79,9 +80,11 @@ __device__ __forceinline__ UnitInfo unit_info(const ModelView &mv, const BatchVi
 
 // ---- launchers implemented in the kernel files; each returns the cudaError_t of its launches ----
 
-// warp-level dot-product scoring (any dtype, any prompt length)
+// warp-level dot-product scoring (any dtype, any prompt length).  row_stats [L][Hq][total_q] is scratch that holds
+// (max base-2 logit, 1 / sum of exp2) per prompt row; row_lse (nullable) is the caller-visible natural-log copy.
 cudaError_t launch_score_simt(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
-                              const BatchView &bv, float *scores, float *row_lse, cudaStream_t stream);
+                              const BatchView &bv, float *scores, float2 *row_stats, float *row_lse,
+                              cudaStream_t stream);
 
 cudaError_t launch_select(const Ctx &ctx, const float *scores, const BatchView &bv, int *kept_idx, int *out_len,
                           cudaStream_t stream);

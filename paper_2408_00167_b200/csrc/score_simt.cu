@@ -1,9 +1,12 @@
 // Prompt-guided scoring with plain FMA dot products (fp32 inputs, or prompts shorter than 64 rows).
 //
 //   lse_simt     one CTA per (64 prompt rows of one query head, unit): sweeps every candidate key and keeps an
-//                online (max, sum-exp) per row -> row_lse
+//                online (max, sum-exp) per row -> row_stats = (max of the base-2 logits, 1 / sum), row_lse
 //   colsum_simt  one CTA per (64 candidate keys, unit): sweeps every prompt row of every head of the group and
-//                accumulates exp(s - lse) per key -> scores
+//                accumulates exp2(s2 - max) / sum per key -> scores
+//
+// Keeping the row maximum and the reciprocal sum apart (instead of one log-sum-exp) keeps the exponent's argument
+// an exact-ish small difference even when the logits are large.
 //
 // A unit is one (layer, selection group, request).  Both kernels tile the logits 64 x 64 with a 4 x 4 register
 // micro-tile per thread and walk head_dim in slices of 32 staged through shared memory.  All sums have a fixed
@@ -73,7 +76,8 @@ __device__ __forceinline__ void fma_slice(float (&acc)[4][4], const float (*qs)[
 
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
-lse_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, TensorView chunk_k, float *row_lse, int *status) {
+lse_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, TensorView chunk_k, float2 *row_stats,
+         float *row_lse, int *status) {
     __shared__ float qs[kTile][kSlice + 1];
     __shared__ float ks[kTile][kSlice + 1];
     const UnitInfo u = unit_info(mv, bv, blockIdx.y, blockIdx.z);
@@ -135,15 +139,18 @@ lse_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, TensorVie
             mx = nmx;
         }
         const int p = p0 + ty + 16 * i;
-        if (tx == 0 && p < u.n_q)
-            row_lse[((int64_t)u.l * mv.Hq + h) * bv.total_q + u.q0 + p] = (mx + log2f(sm)) * kLn2;
+        if (tx == 0 && p < u.n_q) {
+            const int64_t row = ((int64_t)u.l * mv.Hq + h) * bv.total_q + u.q0 + p;
+            row_stats[row] = make_float2(mx, 1.0f / sm);
+            if (row_lse) row_lse[row] = (mx + log2f(sm)) * kLn2;
+        }
     }
 }
 
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
-colsum_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, TensorView chunk_k, const float *row_lse,
-            float *scores, int *status) {
+colsum_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, TensorView chunk_k,
+            const float2 *row_stats, float *scores, int *status) {
     __shared__ float qs[kTile][kSlice + 1];
     __shared__ float ks[kTile][kSlice + 1];
     __shared__ float red[16][kTile];
@@ -160,7 +167,7 @@ colsum_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, Tensor
     float col[4] = {0.f, 0.f, 0.f, 0.f};
     for (int hh = 0; hh < mv.hpg; ++hh) {
         const int h = u.G * mv.hpg + hh, kvh = h / mv.g;
-        const float *lse = row_lse + ((int64_t)u.l * mv.Hq + h) * bv.total_q + u.q0;
+        const float2 *stats = row_stats + ((int64_t)u.l * mv.Hq + h) * bv.total_q + u.q0;
         for (int p0 = 0; p0 < u.n_q; p0 += kTile) {
             float acc[4][4] = {};
             for (int t0 = 0; t0 < mv.d; t0 += kSlice) {
@@ -174,9 +181,9 @@ colsum_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, Tensor
             for (int i = 0; i < 4; ++i) {
                 const int p = p0 + ty + 16 * i;
                 if (p >= u.n_q) continue;
-                const float lse2 = lse[p] * kLog2e;
+                const float2 st = stats[p];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) col[j] += exp2f(acc[i][j] * scale2 - lse2);
+                for (int j = 0; j < 4; ++j) col[j] = fmaf(exp2f(acc[i][j] * scale2 - st.x), st.y, col[j]);
             }
         }
     }
@@ -195,25 +202,28 @@ colsum_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, Tensor
 
 template <typename T>
 cudaError_t launch_t(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
-                     const BatchView &bv, float *scores, float *row_lse, cudaStream_t stream) {
+                     const BatchView &bv, float *scores, float2 *row_stats, float *row_lse, cudaStream_t stream) {
     const ModelView &mv = ctx.model;
     const int units = mv.L * mv.G;
     const int row_blocks = (bv.max_q + kTile - 1) / kTile;
     const int key_tiles = (bv.max_cache + bv.max_chunk + kTile - 1) / kTile;
     if (units == 0 || bv.batch == 0 || row_blocks == 0 || key_tiles == 0) return cudaSuccess;
     dim3 g1(row_blocks * mv.hpg, units, bv.batch);
-    lse_simt<T><<<g1, kThreads, 0, stream>>>(mv, bv, q, cache_k, chunk_k, row_lse, ctx.d_status);
+    lse_simt<T><<<g1, kThreads, 0, stream>>>(mv, bv, q, cache_k, chunk_k, row_stats, row_lse, ctx.d_status);
     dim3 g2(key_tiles, units, bv.batch);
-    colsum_simt<T><<<g2, kThreads, 0, stream>>>(mv, bv, q, cache_k, chunk_k, row_lse, scores, ctx.d_status);
+    colsum_simt<T><<<g2, kThreads, 0, stream>>>(mv, bv, q, cache_k, chunk_k, row_stats, scores, ctx.d_status);
+    ctx.launches += 2;
     return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_score_simt(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
-                              const BatchView &bv, float *scores, float *row_lse, cudaStream_t stream) {
-    if (ctx.cfg.dtype == FINCH_F32) return launch_t<float>(ctx, q, cache_k, chunk_k, bv, scores, row_lse, stream);
-    return launch_t<__nv_bfloat16>(ctx, q, cache_k, chunk_k, bv, scores, row_lse, stream);
+                              const BatchView &bv, float *scores, float2 *row_stats, float *row_lse,
+                              cudaStream_t stream) {
+    if (ctx.cfg.dtype == FINCH_F32)
+        return launch_t<float>(ctx, q, cache_k, chunk_k, bv, scores, row_stats, row_lse, stream);
+    return launch_t<__nv_bfloat16>(ctx, q, cache_k, chunk_k, bv, scores, row_stats, row_lse, stream);
 }
 
 }  // namespace finch

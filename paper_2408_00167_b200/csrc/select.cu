@@ -156,6 +156,7 @@ cudaError_t launch_select(const Ctx &ctx, const float *scores, const BatchView &
     if (e != cudaSuccess) return e;
     dim3 grid(units, bv.batch);
     select_kernel<<<grid, kSelThreads, smem, stream>>>(mv, bv, scores, kept_idx, out_len, smem_keys, ctx.d_status);
+    ctx.launches += 1;
     return cudaGetLastError();
 }
 

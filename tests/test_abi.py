@@ -1,0 +1,157 @@
+"""Host-side checks of the C ABI that need no GPU: exported symbols, argument validation, workspace sizing.
+
+A context created with device = -1 validates arguments exactly like a real one and then refuses to enqueue
+(FINCH_ERR_UNSUPPORTED), so every error path below runs without touching a device.
+"""
+import ctypes as C
+import re
+from pathlib import Path
+
+import pytest
+
+from paper_2408_00167_b200 import binding as fb
+from paper_2408_00167_b200 import build as fbuild
+
+ROOT = Path(__file__).resolve().parents[1]
+
+
+@pytest.fixture(scope="module")
+def lib():
+    fbuild.build()
+    return fb.load()
+
+
+def test_library_exports_every_declared_symbol(lib):
+    header = (ROOT / "include" / "finch.h").read_text()
+    declared = set(re.findall(r"\b(finch_[a-z_]+)\s*\(", header))
+    assert declared == set(fb.EXPORTS)
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def test_status_strings(lib):
+    seen = {fb.finch_status_string(s) for s in range(8)}
+    assert len(seen) == 8 and "ok" in seen
+    assert fb.finch_status_string(99) == "unknown status"
+
+
+def _cfg(**kw):
+    base = dict(n_layers=2, n_q_heads=8, n_kv_heads=2, head_dim=64, dtype=fb.FINCH_BF16,
+                group_mode=fb.FINCH_GROUP_PER_KV_HEAD, scale=0.0, max_batch=4, max_prompt=64, max_candidates=1024,
+                device=-1)
+    base.update(kw)
+    return base
+
+
+@pytest.mark.parametrize("bad,status", [
+    (dict(n_layers=0), fb.FINCH_ERR_INVALID_ARG),
+    (dict(n_q_heads=6, n_kv_heads=4), fb.FINCH_ERR_INVALID_ARG),
+    (dict(dtype=7), fb.FINCH_ERR_INVALID_ARG),
+    (dict(group_mode=3), fb.FINCH_ERR_INVALID_ARG),
+    (dict(scale=-1.0), fb.FINCH_ERR_INVALID_ARG),
+    (dict(scale=float("nan")), fb.FINCH_ERR_INVALID_ARG),
+    (dict(max_batch=0), fb.FINCH_ERR_INVALID_ARG),
+    (dict(head_dim=48), fb.FINCH_ERR_UNSUPPORTED),
+    (dict(head_dim=512), fb.FINCH_ERR_UNSUPPORTED),
+])
+def test_ctx_create_rejects_bad_configs(lib, bad, status):
+    with pytest.raises(fb.FinchError) as e:
+        fb.finch_ctx_create(**_cfg(**bad))
+    assert e.value.status == status
+
+
+def test_ctx_create_null_arguments(lib):
+    assert lib.finch_ctx_create(None, None) == fb.FINCH_ERR_INVALID_ARG
+    lib.finch_ctx_destroy(None)   # ignored
+
+
+def test_real_device_is_refused_without_a_b200(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    with pytest.raises(fb.FinchError) as e:
+        fb.finch_ctx_create(**_cfg(device=0))
+    assert e.value.status == fb.FINCH_ERR_UNSUPPORTED
+
+
+class _Fake:
+    """Stand-ins for device buffers: validation only looks at addresses, never dereferences them."""
+    base = 0x7000_0000_0000
+
+    @classmethod
+    def batch(cls, B=2, total_q=96, total_chunk=512, total_cache=256, max_q=64, max_cache=128, max_chunk=256,
+              max_budget=128):
+        p = cls.base
+        return fb.Batch(None, None, None, None, None,
+                        fb.finch_batch(B, p, p + 256, p + 512, p + 768, p + 1024, total_q, total_chunk, total_cache,
+                                       max_q, max_cache, max_chunk, max_budget))
+
+    @classmethod
+    def tensor(cls, slot, tokens, d=64, heads=2, misalign=0, stride_tok=None):
+        st = d if stride_tok is None else stride_tok
+        return fb.finch_tensor(cls.base + 0x1000_0000 * (slot + 1) + misalign, heads * tokens * st, tokens * st, st)
+
+
+def _step(lib, ctx, batch, q=None, ck=None, cv=None, hk=None, hv=None, ok=None, ov=None, ws=_Fake.base + 0x9000_0000,
+          ws_bytes=1 << 30, scores=None, kept=_Fake.base + 0xA000_0000, out_len=_Fake.base + 0xA100_0000,
+          cache_pos=_Fake.base + 0xA200_0000, chunk_pos=_Fake.base + 0xA300_0000, out_pos=_Fake.base + 0xA400_0000):
+    c = batch.c
+    q = q or _Fake.tensor(0, c.total_q, heads=8)
+    ck, cv = ck or _Fake.tensor(1, c.total_cache), cv or _Fake.tensor(2, c.total_cache)
+    hk, hv = hk or _Fake.tensor(3, c.total_chunk), hv or _Fake.tensor(4, c.total_chunk)
+    ok, ov = ok or _Fake.tensor(5, c.total_cache), ov or _Fake.tensor(6, c.total_cache)
+    return lib.finch_step(ctx, C.byref(q), C.byref(ck), C.byref(cv), C.c_void_p(cache_pos), C.byref(hk), C.byref(hv),
+                          C.c_void_p(chunk_pos), C.byref(c), C.byref(ok), C.byref(ov), C.c_void_p(out_pos),
+                          C.c_void_p(kept), C.c_void_p(out_len), C.c_void_p(scores), C.c_void_p(ws),
+                          C.c_size_t(ws_bytes), None)
+
+
+def test_step_validation_paths(lib):
+    ctx = fb.finch_ctx_create(**_cfg())
+    try:
+        good = _Fake.batch()
+        # a fully valid call reaches the launch stage, where a validation-only context stops
+        assert _step(lib, ctx, good) == fb.FINCH_ERR_UNSUPPORTED
+        assert _step(lib, ctx, good, ws=None) == fb.FINCH_ERR_INVALID_ARG
+        assert _step(lib, ctx, good, ws=_Fake.base + 8) == fb.FINCH_ERR_BAD_LAYOUT
+        assert _step(lib, ctx, good, ws_bytes=16) == fb.FINCH_ERR_WORKSPACE_TOO_SMALL
+        assert _step(lib, ctx, good, kept=None) == fb.FINCH_ERR_INVALID_ARG
+        assert _step(lib, ctx, good, out_len=None) == fb.FINCH_ERR_INVALID_ARG
+        assert _step(lib, ctx, good, cache_pos=None) == fb.FINCH_ERR_INVALID_ARG
+        assert _step(lib, ctx, good, chunk_pos=None) == fb.FINCH_ERR_INVALID_ARG
+        assert _step(lib, ctx, good, q=_Fake.tensor(0, 96, heads=8, misalign=4)) == fb.FINCH_ERR_BAD_LAYOUT
+        assert _step(lib, ctx, good, hk=_Fake.tensor(3, 512, stride_tok=68)) == fb.FINCH_ERR_BAD_LAYOUT
+        assert _step(lib, ctx, good, hk=_Fake.tensor(3, 512, stride_tok=32)) == fb.FINCH_ERR_INVALID_ARG
+        # outputs may not alias inputs (parallel gather)
+        assert _step(lib, ctx, good, ok=_Fake.tensor(1, 256)) == fb.FINCH_ERR_INVALID_ARG
+        assert _step(lib, ctx, good, ov=_Fake.tensor(5, 256)) == fb.FINCH_ERR_INVALID_ARG
+        # batch bounds against the context and against themselves
+        assert _step(lib, ctx, _Fake.batch(B=5)) == fb.FINCH_ERR_INVALID_ARG
+        assert _step(lib, ctx, _Fake.batch(max_q=65, total_q=128)) == fb.FINCH_ERR_INVALID_ARG
+        assert _step(lib, ctx, _Fake.batch(max_cache=900, total_cache=900, max_chunk=256)) == fb.FINCH_ERR_INVALID_ARG
+        assert _step(lib, ctx, _Fake.batch(max_q=0)) == fb.FINCH_ERR_INVALID_ARG
+        assert _step(lib, ctx, _Fake.batch(max_budget=300)) == fb.FINCH_ERR_INVALID_ARG
+        nullb = _Fake.batch()
+        nullb.c.q_off = None
+        assert _step(lib, ctx, nullb) == fb.FINCH_ERR_INVALID_ARG
+    finally:
+        fb.finch_ctx_destroy(ctx)
+
+
+def test_workspace_bytes_is_host_arithmetic(lib):
+    ctx = fb.finch_ctx_create(**_cfg())
+    try:
+        b = _Fake.batch()
+        n = fb.finch_workspace_bytes(ctx, b)
+        lse = 2 * 8 * 96 * 8
+        scores = 2 * 2 * (256 + 512) * 4
+        assert n >= lse + scores and n % 256 == 0
+        bigger = _Fake.batch(total_q=192)
+        assert fb.finch_workspace_bytes(ctx, bigger) > n
+        out = C.c_size_t()
+        assert lib.finch_workspace_bytes(ctx, C.byref(b.c), None) == fb.FINCH_ERR_INVALID_ARG
+        assert lib.finch_workspace_bytes(None, C.byref(b.c), C.byref(out)) == fb.FINCH_ERR_INVALID_ARG
+        status = C.c_int32()
+        assert lib.finch_device_status(ctx, None, C.byref(status)) == fb.FINCH_ERR_UNSUPPORTED
+    finally:
+        fb.finch_ctx_destroy(ctx)
