@@ -106,7 +106,7 @@ def aggregate_over_ranks(ms_local: float, tokens_local: int, world: int, backend
     return float(t.item()), int(n.item())
 
 
-def oracle_sample(cfg: wl.Config, target_s: float = 12.0, max_layers: int = 4):
+def oracle_sample(cfg: wl.Config, target_s: float = 12.0, max_layers: int = 32):
     """Time the fp64 oracle's whole step on whole layers of the same workload until about target_s of CPU work."""
     import oracle
     threads = oracle.max_threads()

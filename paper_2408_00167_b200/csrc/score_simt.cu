@@ -6,7 +6,8 @@
 //                accumulates exp2(s2 - max) / sum per key -> scores
 //
 // Keeping the row maximum and the reciprocal sum apart (instead of one log-sum-exp) keeps the exponent's argument
-// an exact-ish small difference even when the logits are large.
+// a small difference even when the logits are large; both kernels form it with the same fused multiply-add
+// (dot * scale2 - max), so the weight of a row's largest key is the same in the sum and in the column pass.
 //
 // A unit is one (layer, selection group, request).  Both kernels tile the logits 64 x 64 with a 4 x 4 register
 // micro-tile per thread and walk head_dim in slices of 32 staged through shared memory.  All sums have a fixed
@@ -119,7 +120,7 @@ lse_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, TensorVie
             float sum = run_sum[i] * exp2f(run_max[i] - new_max);  // exp2(-inf) = 0 on the first tile
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-                if (j0 + tx + 16 * j < u.N) sum += exp2f(acc[i][j] * scale2 - new_max);
+                if (j0 + tx + 16 * j < u.N) sum += exp2f(fmaf(acc[i][j], scale2, -new_max));
             run_max[i] = new_max;
             run_sum[i] = sum;
         }
@@ -183,7 +184,7 @@ colsum_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, Tensor
                 if (p >= u.n_q) continue;
                 const float2 st = stats[p];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) col[j] = fmaf(exp2f(acc[i][j] * scale2 - st.x), st.y, col[j]);
+                for (int j = 0; j < 4; ++j) col[j] = fmaf(exp2f(fmaf(acc[i][j], scale2, -st.x)), st.y, col[j]);
             }
         }
     }

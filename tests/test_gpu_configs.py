@@ -99,7 +99,10 @@ def _select_only(scores_np, chunk_lens, cache_caps, cache_lens, budgets, L, G):
     ctx = fb.finch_ctx_create(L, G, G, 64, fb.FINCH_F32, max_batch=B, max_prompt=1,
                               max_candidates=max(c.max_cache + c.max_chunk, 1))
     try:
-        scores = torch.from_numpy(scores_np).cuda()
+        # the score rows are laid out with the full candidate stride (cache capacity + chunk rows)
+        padded = np.full((L, G, c.total_cache + c.total_chunk), np.nan, np.float32)
+        padded[:, :, :scores_np.shape[2]] = scores_np
+        scores = torch.from_numpy(padded).cuda()
         kept = torch.full((L, G, c.total_cache), -1, dtype=torch.int32, device="cuda")
         out_len = torch.zeros(B, dtype=torch.int32, device="cuda")
         fb.finch_select(ctx, scores, batch, kept, out_len)
