@@ -137,6 +137,27 @@ finch_status finch_score(finch_ctx *ctx, const finch_tensor *prompt_q, const fin
                          const finch_tensor *chunk_k, const finch_batch *batch, float *scores, float *row_lse,
                          void *ws, size_t ws_bytes, void *cuda_stream);
 
+/* Same computation and outputs as finch_score, for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is an integration aid.)  Some hosts of this library may not call cudaMalloc at all -- a plugin
+ * inside a serving process whose memory pool owns the whole device, or a step that must stay clear of the driver's
+ * allocator for latency reasons -- and so cannot supply finch_score's workspace.  Here the per-row softmax
+ * statistics that finch_score keeps in that workspace live in a fixed array inside the library image instead
+ * (8 MiB of device memory on every GPU that loads the library, held until the process exits).  The call itself
+ * allocates and frees nothing.
+ *  - Limit: n_layers * n_q_heads * total_q must not exceed finch_score_static_max_rows() (2^20 rows); a larger
+ *    batch is rejected with FINCH_ERR_WORKSPACE_TOO_SMALL and nothing is enqueued -- use finch_score then.
+ *  - The first call on each device looks up the array's device address; the context's device must be the current
+ *    device (FINCH_ERR_INVALID_ARG otherwise).  Make that first call before starting any stream capture.
+ *  - Every call on a device shares the one array, which keeps the previous call's contents.  Nothing in it has
+ *    to start at zero: each call overwrites every entry it later reads.  Two calls whose kernels overlap on the
+ *    GPU (different streams, or different contexts on one device) race on it: serialise them. */
+finch_status finch_score_static(finch_ctx *ctx, const finch_tensor *prompt_q, const finch_tensor *cache_k,
+                                const finch_tensor *chunk_k, const finch_batch *batch, float *scores, float *row_lse,
+                                void *cuda_stream);
+
+/* The row limit of finch_score_static. */
+size_t finch_score_static_max_rows(void);
+
 /* Top-r selection (Method, bullet "Selection of top r position": t = top-r(A^agg, r)).  For every layer, group and
  * request keeps r' = min(budget[b], N_b) candidates with the largest scores; among equal scores the lower
  * candidate index wins; -0 equals +0; a NaN ranks below every number.  Writes the kept candidate indices in

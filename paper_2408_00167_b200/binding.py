@@ -29,7 +29,7 @@ FINCH_GROUP_PER_KV_HEAD, FINCH_GROUP_PER_LAYER = 0, 1
 FINCH_DEV_BAD_BATCH, FINCH_DEV_TIMEOUT, FINCH_DEV_BAD_INDEX = 1, 2, 4
 
 EXPORTS = ("finch_ctx_create", "finch_ctx_destroy", "finch_workspace_bytes", "finch_score", "finch_select",
-           "finch_compact", "finch_step", "finch_device_status", "finch_launch_count", "finch_status_string")
+           "finch_compact", "finch_step", "finch_device_status", "finch_launch_count", "finch_status_string", "finch_score_static", "finch_score_static_max_rows")
 
 
 class finch_config(C.Structure):
@@ -68,6 +68,7 @@ def load() -> C.CDLL:
             getattr(lib, name).restype = C.c_int
         lib.finch_ctx_destroy.restype = None
         lib.finch_status_string.restype = C.c_char_p
+        lib.finch_score_static_max_rows.restype = C.c_size_t
         _lib = lib
     return _lib
 
@@ -211,3 +212,16 @@ def finch_launch_count(ctx) -> int:
     out = C.c_uint64()
     _check(load().finch_launch_count(ctx, C.byref(out)), "finch_launch_count")
     return int(out.value)
+
+
+def finch_score_static(ctx, prompt_q, cache_k, chunk_k, batch: Batch, scores, row_lse=None, stream=None) -> None:
+    """finch_score without a workspace: the scratch is a fixed array inside the library (see finch.h for the
+    row limit and the sharing rules).  For callers that may not allocate device memory."""
+    q, ck, hk = _tensor(prompt_q), _tensor(cache_k), _tensor(chunk_k)
+    _check(load().finch_score_static(ctx, C.byref(q), C.byref(ck), C.byref(hk), C.byref(batch.c),
+                                     C.c_void_p(_ptr(scores)), C.c_void_p(_ptr(row_lse)),
+                                     C.c_void_p(_stream(stream))), "finch_score_static")
+
+
+def finch_score_static_max_rows() -> int:
+    return int(load().finch_score_static_max_rows())

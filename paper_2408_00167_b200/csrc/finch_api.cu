@@ -281,3 +281,60 @@ finch_status finch_device_status(finch_ctx *ctx, void *cuda_stream, int32_t *out
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------------------------
+// finch_score_static: scoring for callers that cannot allocate device memory.
+//
+// finch_score keeps one (row maximum, 1 / row sum) pair per prompt row between its two kernels, in a workspace the
+// caller allocates.  Code that runs where cudaMalloc is off limits -- a plugin inside a serving process that owns
+// all device memory and hands none out, a callback that may not block on the allocator, a latency-critical loop
+// that must not touch the driver's heap -- has no such workspace to give.  For those callers the pairs live in the
+// fixed array below, which is part of the library image: every GPU that loads libfinch holds it until the process
+// exits.
+namespace {
+
+constexpr size_t kStaticRows = size_t(1) << 20;  // prompt rows (layers x query heads x packed prompt tokens): 8 MiB
+static __device__ __align__(256) float2 g_static_row_stats[kStaticRows];
+
+constexpr int kMaxDevices = 64;
+float2 *g_static_ptr[kMaxDevices] = {};  // device address of the array on each device, filled on first use
+
+// In host code the array's name is only a handle; its device address has to be asked for, once per device, with
+// that device current.
+finch_status static_scratch(int device, float2 **out) {
+    if (device < 0 || device >= kMaxDevices) return FINCH_ERR_UNSUPPORTED;
+    if (!g_static_ptr[device]) {
+        int current = -1;
+        if (cudaGetDevice(&current) != cudaSuccess || current != device) {
+            (void)cudaGetLastError();
+            return FINCH_ERR_INVALID_ARG;  // the context's device must be the current one
+        }
+        float2 *p = nullptr;
+        if (cudaGetSymbolAddress((void **)&p, g_static_row_stats) != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return FINCH_ERR_CUDA;
+        }
+        g_static_ptr[device] = p;
+    }
+    *out = g_static_ptr[device];
+    return FINCH_OK;
+}
+
+}  // namespace
+
+extern "C" finch_status finch_score_static(finch_ctx *ctx, const finch_tensor *prompt_q, const finch_tensor *cache_k,
+                                           const finch_tensor *chunk_k, const finch_batch *batch, float *scores,
+                                           float *row_lse, void *cuda_stream) {
+    finch_status s = validate_score(ctx, prompt_q, cache_k, chunk_k, batch);
+    if (s) return s;
+    if (!scores && (size_t)batch->total_cache + batch->total_chunk > 0) return FINCH_ERR_INVALID_ARG;
+    const size_t rows = (size_t)ctx->model.L * ctx->model.Hq * (size_t)batch->total_q;
+    if (rows > kStaticRows) return FINCH_ERR_WORKSPACE_TOO_SMALL;  // beyond the built-in scratch: use finch_score
+    if (ctx->dry) return FINCH_ERR_UNSUPPORTED;
+    float2 *row_stats = nullptr;
+    if ((s = static_scratch(ctx->cfg.device, &row_stats))) return s;
+    return cuda_status(launch_score_simt(*ctx, view_of(prompt_q), view_of(cache_k), view_of(chunk_k), view_of(batch),
+                                         scores, row_stats, row_lse, (cudaStream_t)cuda_stream));
+}
+
+extern "C" size_t finch_score_static_max_rows(void) { return kStaticRows; }
