@@ -61,7 +61,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -196,15 +196,14 @@ def run_ours(args, cfg: wl.Config):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / n
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()               # runs through warm-up, the timed steps and the per-phase loop: all under load
     for _ in range(max(args.warmup, 3)):
         step()
     assert fb.finch_device_status(ctx) == 0
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     launches0 = fb.finch_launch_count(ctx)
     ms_local = timed(step, args.steps)
     launches = fb.finch_launch_count(ctx) - launches0
-    clocks = sampler.stop()
     assert fb.finch_device_status(ctx) == 0
     ms, tokens = aggregate_over_ranks(ms_local, counts["tokens"], world, "nccl")
 
@@ -223,6 +222,7 @@ def run_ours(args, cfg: wl.Config):
         torch.cuda.synchronize()
         phase += [ev[i].elapsed_time(ev[i + 1]) for i in range(3)]
     phase /= args.steps
+    clocks = sampler.stop()
 
     step_e2e()
     ms_e2e_local = timed(step_e2e, max(1, min(args.steps, 5)))

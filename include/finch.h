@@ -108,6 +108,7 @@ typedef struct {
     const int32_t *cache_len, *budget;            /* device, [batch]; budget[b] = r, at most the capacity     */
     int32_t total_q, total_chunk, total_cache;    /* host copies of q_off[batch], chunk_off[batch], cache_off[batch] */
     int32_t max_q, max_cache, max_chunk, max_budget; /* host upper bounds over the requests (grid sizing)      */
+    int32_t min_q;                                /* host lower bound of the prompt lengths; 0 when unknown    */
 } finch_batch;
 
 /* Create a context for one model shape on one device.  Fails with FINCH_ERR_UNSUPPORTED when the device is not

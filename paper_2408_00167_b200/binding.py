@@ -48,7 +48,8 @@ class finch_batch(C.Structure):
     _fields_ = [("batch", C.c_int32), ("q_off", C.c_void_p), ("chunk_off", C.c_void_p), ("cache_off", C.c_void_p),
                 ("cache_len", C.c_void_p), ("budget", C.c_void_p), ("total_q", C.c_int32),
                 ("total_chunk", C.c_int32), ("total_cache", C.c_int32), ("max_q", C.c_int32),
-                ("max_cache", C.c_int32), ("max_chunk", C.c_int32), ("max_budget", C.c_int32)]
+                ("max_cache", C.c_int32), ("max_chunk", C.c_int32), ("max_budget", C.c_int32),
+                ("min_q", C.c_int32)]
 
 
 class FinchError(RuntimeError):
@@ -140,7 +141,8 @@ def make_batch(q_off: Sequence[int], chunk_off: Sequence[int], cache_off: Sequen
         return int(a.max()) if len(a) else 0
     n_cand = h[3] + diff(h[1])
     cb = finch_batch(B, *[x.data_ptr() for x in d], int(h[0][B]), int(h[1][B]), int(h[2][B]),
-                     mx(diff(h[0])), mx(h[3]), mx(diff(h[1])), mx(np.minimum(h[4], n_cand)) if B else 0)
+                     mx(diff(h[0])), mx(h[3]), mx(diff(h[1])), mx(np.minimum(h[4], n_cand)) if B else 0,
+                     int(diff(h[0]).min()) if B else 0)
     return Batch(*d, cb)
 
 

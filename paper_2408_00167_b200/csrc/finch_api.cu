@@ -1,4 +1,5 @@
 // Host side of the C ABI: context, argument validation, workspace layout and kernel dispatch.
+#include <limits.h>
 #include <math.h>
 #include <new>
 #include <string.h>
@@ -30,6 +31,7 @@ finch_status check_batch(const finch_ctx *ctx, const finch_batch *b) {
     if (!ctx || !b) return FINCH_ERR_INVALID_ARG;
     if (b->batch < 0 || b->batch > ctx->cfg.max_batch) return FINCH_ERR_INVALID_ARG;
     if (b->total_q < 0 || b->total_chunk < 0 || b->total_cache < 0) return FINCH_ERR_INVALID_ARG;
+    if (b->min_q < 0 || b->min_q > b->max_q) return FINCH_ERR_INVALID_ARG;
     if (b->max_q < 0 || b->max_cache < 0 || b->max_chunk < 0 || b->max_budget < 0) return FINCH_ERR_INVALID_ARG;
     if (b->max_q > ctx->cfg.max_prompt) return FINCH_ERR_INVALID_ARG;
     if ((int64_t)b->max_cache + b->max_chunk > ctx->cfg.max_candidates) return FINCH_ERR_INVALID_ARG;
@@ -102,6 +104,29 @@ finch_status validate_compact(const finch_ctx *ctx, const int32_t *kept_idx, con
 }
 
 }  // namespace
+
+namespace finch {
+
+// Tensor cores take the requests whose prompt has at least 64 rows (bf16, supported head_dim); warp-level dot
+// products take the rest.  batch.min_q lets the host skip the launch that would find no request of its class.
+cudaError_t run_score(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
+                      const BatchView &bv, float *scores, float2 *row_stats, float *row_lse, cudaStream_t stream) {
+    constexpr int kTensorCoreMinRows = 64;
+    int simt_below = INT_MAX;
+    if (score_tc_supported(ctx) && bv.max_q >= kTensorCoreMinRows) {
+        const cudaError_t e = launch_score_tc(ctx, q, cache_k, chunk_k, bv, scores, row_stats, row_lse,
+                                              kTensorCoreMinRows, stream);
+        if (e == cudaSuccess) {
+            if (bv.min_q >= kTensorCoreMinRows) return cudaSuccess;
+            simt_below = kTensorCoreMinRows;
+        } else if (e != cudaErrorNotSupported) {
+            return e;
+        }
+    }
+    return launch_score_simt(ctx, q, cache_k, chunk_k, bv, scores, row_stats, row_lse, simt_below, stream);
+}
+
+}  // namespace finch
 
 extern "C" {
 
@@ -201,8 +226,8 @@ finch_status finch_score(finch_ctx *ctx, const finch_tensor *prompt_q, const fin
     if (ws_bytes < w.lse_off + w.lse_bytes) return FINCH_ERR_WORKSPACE_TOO_SMALL;
     float2 *row_stats = (float2 *)((char *)ws + w.lse_off);
     if (ctx->dry) return FINCH_ERR_UNSUPPORTED;
-    return cuda_status(launch_score_simt(*ctx, view_of(prompt_q), view_of(cache_k), view_of(chunk_k), view_of(batch),
-                                         scores, row_stats, row_lse, (cudaStream_t)cuda_stream));
+    return cuda_status(run_score(*ctx, view_of(prompt_q), view_of(cache_k), view_of(chunk_k), view_of(batch), scores,
+                                 row_stats, row_lse, (cudaStream_t)cuda_stream));
 }
 
 finch_status finch_select(finch_ctx *ctx, const float *scores, const finch_batch *batch, int32_t *kept_idx,
@@ -250,8 +275,8 @@ finch_status finch_step(finch_ctx *ctx, const finch_tensor *prompt_q, const finc
     if (ctx->dry) return FINCH_ERR_UNSUPPORTED;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     const BatchView bv = view_of(batch);
-    cudaError_t e = launch_score_simt(*ctx, view_of(prompt_q), view_of(cache_k), view_of(chunk_k), bv, scores, row_stats,
-                                      nullptr, stream);
+    cudaError_t e = run_score(*ctx, view_of(prompt_q), view_of(cache_k), view_of(chunk_k), bv, scores, row_stats,
+                              nullptr, stream);
     if (e == cudaSuccess) e = launch_select(*ctx, scores, bv, kept_idx, out_len, stream);
     if (e == cudaSuccess)
         e = launch_compact(*ctx, kept_idx, out_len, view_of(cache_k), view_of(cache_v), cache_pos, view_of(chunk_k),
@@ -333,8 +358,8 @@ extern "C" finch_status finch_score_static(finch_ctx *ctx, const finch_tensor *p
     if (ctx->dry) return FINCH_ERR_UNSUPPORTED;
     float2 *row_stats = nullptr;
     if ((s = static_scratch(ctx->cfg.device, &row_stats))) return s;
-    return cuda_status(launch_score_simt(*ctx, view_of(prompt_q), view_of(cache_k), view_of(chunk_k), view_of(batch),
-                                         scores, row_stats, row_lse, (cudaStream_t)cuda_stream));
+    return cuda_status(run_score(*ctx, view_of(prompt_q), view_of(cache_k), view_of(chunk_k), view_of(batch), scores,
+                                 row_stats, row_lse, (cudaStream_t)cuda_stream));
 }
 
 extern "C" size_t finch_score_static_max_rows(void) { return kStaticRows; }

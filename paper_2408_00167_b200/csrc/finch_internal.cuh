@@ -20,6 +20,7 @@ struct BatchView {
     const int *q_off, *chunk_off, *cache_off, *cache_len, *budget;
     int total_q, total_chunk, total_cache;
     int max_q, max_cache, max_chunk, max_budget;
+    int min_q;
 };
 
 struct ModelView {
@@ -46,7 +47,8 @@ inline TensorView view_of(const finch_tensor *t) {
 }
 inline BatchView view_of(const finch_batch *b) {
     return BatchView{b->batch,       b->q_off,       b->chunk_off, b->cache_off, b->cache_len, b->budget,    b->total_q,
-                     b->total_chunk, b->total_cache, b->max_q,     b->max_cache, b->max_chunk, b->max_budget};
+                     b->total_chunk, b->total_cache, b->max_q,     b->max_cache, b->max_chunk, b->max_budget,
+                     b->min_q};
 }
 
 constexpr float kLog2e = 1.4426950408889634f;
@@ -83,8 +85,18 @@ __device__ __forceinline__ UnitInfo unit_info(const ModelView &mv, const BatchVi
 // warp-level dot-product scoring (any dtype, any prompt length).  row_stats [L][Hq][total_q] is scratch that holds
 // (max base-2 logit, 1 / sum of exp2) per prompt row; row_lse (nullable) is the caller-visible natural-log copy.
 cudaError_t launch_score_simt(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
-                              const BatchView &bv, float *scores, float2 *row_stats, float *row_lse,
+                              const BatchView &bv, float *scores, float2 *row_stats, float *row_lse, int nq_below,
                               cudaStream_t stream);
+
+// tensor-core scoring (bf16, head_dim 64 or 128, one KV head per group) for requests with n_q >= min_q
+bool score_tc_supported(const Ctx &ctx);
+cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
+                            const BatchView &bv, float *scores, float2 *row_stats, float *row_lse, int min_q,
+                            cudaStream_t stream);
+
+// scoring dispatch shared by finch_score, finch_score_static and finch_step
+cudaError_t run_score(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
+                      const BatchView &bv, float *scores, float2 *row_stats, float *row_lse, cudaStream_t stream);
 
 cudaError_t launch_select(const Ctx &ctx, const float *scores, const BatchView &bv, int *kept_idx, int *out_len,
                           cudaStream_t stream);

@@ -84,7 +84,7 @@ class _Fake:
         p = cls.base
         return fb.Batch(None, None, None, None, None,
                         fb.finch_batch(B, p, p + 256, p + 512, p + 768, p + 1024, total_q, total_chunk, total_cache,
-                                       max_q, max_cache, max_chunk, max_budget))
+                                       max_q, max_cache, max_chunk, max_budget, 0))
 
     @classmethod
     def tensor(cls, slot, tokens, d=64, heads=2, misalign=0, stride_tok=None):

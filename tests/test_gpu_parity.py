@@ -56,6 +56,9 @@ SHAPES = [
     ("bf16", 8, 2, 128, [(16, 9999, 200, 100)]),
     ("bf16", 4, 4, 64, [(63, 9999, 129, 64)]),
     ("bf16", 8, 2, 128, [(5, 9999, 64, 17), (33, 9999, 100, 300), (20, 9999, 1, 1)]),
+    # tensor-core path (>= 64 prompt rows): partial row blocks, partial key tiles on both sides of the cache/chunk seam
+    ("bf16", 8, 2, 128, [(130, 9999, 300, 333)]),
+    ("bf16", 4, 2, 64, [(64, 9999, 1, 129), (257, 9999, 257, 255), (40, 9999, 90, 70)]),
 ]
 
 
