@@ -287,8 +287,11 @@ def main():
     ap.add_argument("--config", default="c3", choices=sorted(wl.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (small profiling runs)")
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.config]
+    if args.layers > 0:
+        cfg = wl.scaled(cfg, n_layers=min(args.layers, cfg.n_layers))
     if args.impl == "reference":
         line = run_reference(args, cfg)
     else:

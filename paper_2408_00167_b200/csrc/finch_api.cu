@@ -44,7 +44,7 @@ finch_status check_batch(const finch_ctx *ctx, const finch_batch *b) {
 }
 
 struct WsLayout {
-    size_t lse_off, lse_bytes;        // per prompt row (max, 1/sum) of the softmax, float2
+    size_t lse_off, lse_bytes;        // softmax statistics: one float2 per prompt row and key split
     size_t scores_off, scores_bytes;  // scores inside finch_step when the caller gives none
     size_t total;
 };
@@ -53,7 +53,7 @@ WsLayout ws_layout(const finch_ctx *ctx, const finch_batch *b) {
     WsLayout w{};
     const ModelView &mv = ctx->model;
     w.lse_off = 0;
-    w.lse_bytes = align_up((size_t)mv.L * mv.Hq * (size_t)b->total_q * sizeof(float2));
+    w.lse_bytes = align_up((size_t)mv.L * mv.Hq * (size_t)b->total_q * sizeof(float2) * kScoreMaxSplits * 2);
     w.scores_off = w.lse_off + w.lse_bytes;
     w.scores_bytes = align_up((size_t)mv.L * mv.G * ((size_t)b->total_cache + b->total_chunk) * sizeof(float));
     w.total = w.scores_off + w.scores_bytes;
@@ -110,11 +110,12 @@ namespace finch {
 // Tensor cores take the requests whose prompt has at least 64 rows (bf16, supported head_dim); warp-level dot
 // products take the rest.  batch.min_q lets the host skip the launch that would find no request of its class.
 cudaError_t run_score(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
-                      const BatchView &bv, float *scores, float2 *row_stats, float *row_lse, cudaStream_t stream) {
+                      const BatchView &bv, float *scores, float2 *scratch, size_t scratch_capacity, float *row_lse,
+                      cudaStream_t stream) {
     constexpr int kTensorCoreMinRows = 64;
     int simt_below = INT_MAX;
     if (score_tc_supported(ctx) && bv.max_q >= kTensorCoreMinRows) {
-        const cudaError_t e = launch_score_tc(ctx, q, cache_k, chunk_k, bv, scores, row_stats, row_lse,
+        const cudaError_t e = launch_score_tc(ctx, q, cache_k, chunk_k, bv, scores, scratch, scratch_capacity, row_lse,
                                               kTensorCoreMinRows, stream);
         if (e == cudaSuccess) {
             if (bv.min_q >= kTensorCoreMinRows) return cudaSuccess;
@@ -123,7 +124,7 @@ cudaError_t run_score(const Ctx &ctx, const TensorView &q, const TensorView &cac
             return e;
         }
     }
-    return launch_score_simt(ctx, q, cache_k, chunk_k, bv, scores, row_stats, row_lse, simt_below, stream);
+    return launch_score_simt(ctx, q, cache_k, chunk_k, bv, scores, scratch, row_lse, simt_below, stream);
 }
 
 }  // namespace finch
@@ -227,7 +228,7 @@ finch_status finch_score(finch_ctx *ctx, const finch_tensor *prompt_q, const fin
     float2 *row_stats = (float2 *)((char *)ws + w.lse_off);
     if (ctx->dry) return FINCH_ERR_UNSUPPORTED;
     return cuda_status(run_score(*ctx, view_of(prompt_q), view_of(cache_k), view_of(chunk_k), view_of(batch), scores,
-                                 row_stats, row_lse, (cudaStream_t)cuda_stream));
+                                 row_stats, w.lse_bytes / sizeof(float2), row_lse, (cudaStream_t)cuda_stream));
 }
 
 finch_status finch_select(finch_ctx *ctx, const float *scores, const finch_batch *batch, int32_t *kept_idx,
@@ -276,7 +277,7 @@ finch_status finch_step(finch_ctx *ctx, const finch_tensor *prompt_q, const finc
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     const BatchView bv = view_of(batch);
     cudaError_t e = run_score(*ctx, view_of(prompt_q), view_of(cache_k), view_of(chunk_k), bv, scores, row_stats,
-                              nullptr, stream);
+                              w.lse_bytes / sizeof(float2), nullptr, stream);
     if (e == cudaSuccess) e = launch_select(*ctx, scores, bv, kept_idx, out_len, stream);
     if (e == cudaSuccess)
         e = launch_compact(*ctx, kept_idx, out_len, view_of(cache_k), view_of(cache_v), cache_pos, view_of(chunk_k),
@@ -359,7 +360,7 @@ extern "C" finch_status finch_score_static(finch_ctx *ctx, const finch_tensor *p
     float2 *row_stats = nullptr;
     if ((s = static_scratch(ctx->cfg.device, &row_stats))) return s;
     return cuda_status(run_score(*ctx, view_of(prompt_q), view_of(cache_k), view_of(chunk_k), view_of(batch), scores,
-                                 row_stats, row_lse, (cudaStream_t)cuda_stream));
+                                 row_stats, kStaticRows, row_lse, (cudaStream_t)cuda_stream));
 }
 
 extern "C" size_t finch_score_static_max_rows(void) { return kStaticRows; }

@@ -88,15 +88,19 @@ cudaError_t launch_score_simt(const Ctx &ctx, const TensorView &q, const TensorV
                               const BatchView &bv, float *scores, float2 *row_stats, float *row_lse, int nq_below,
                               cudaStream_t stream);
 
-// tensor-core scoring (bf16, head_dim 64 or 128, one KV head per group) for requests with n_q >= min_q
+// tensor-core scoring (bf16, head_dim 64 or 128, one KV head per group) for requests with n_q >= min_q.  The scratch
+// holds one float2 per prompt row and key split; up to kScoreMaxSplits splits are used when it is large enough.
+constexpr int kScoreMaxSplits = 8;
 bool score_tc_supported(const Ctx &ctx);
 cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
-                            const BatchView &bv, float *scores, float2 *row_stats, float *row_lse, int min_q,
-                            cudaStream_t stream);
+                            const BatchView &bv, float *scores, float2 *partial, size_t partial_capacity,
+                            float *row_lse, int min_q, cudaStream_t stream);
 
-// scoring dispatch shared by finch_score, finch_score_static and finch_step
+// scoring dispatch shared by finch_score, finch_score_static and finch_step; `scratch` holds scratch_capacity
+// float2 entries, at least one per prompt row (n_layers * n_q_heads * total_q)
 cudaError_t run_score(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
-                      const BatchView &bv, float *scores, float2 *row_stats, float *row_lse, cudaStream_t stream);
+                      const BatchView &bv, float *scores, float2 *scratch, size_t scratch_capacity, float *row_lse,
+                      cudaStream_t stream);
 
 cudaError_t launch_select(const Ctx &ctx, const float *scores, const BatchView &bv, int *kept_idx, int *out_len,
                           cudaStream_t stream);

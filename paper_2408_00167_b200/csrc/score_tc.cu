@@ -1,19 +1,21 @@
 // Prompt-guided scoring on the 5th-generation tensor cores (bf16 inputs, prompts of at least 64 rows).
 //
-// One kernel template, two sweeps over the logits S = Q K^T of a unit (layer, KV head, request):
+// One kernel template, two sweeps over the logits S = Q K^T of a unit (layer, KV head, request).  A CTA owns one
+// split of the unit's 128-key tiles and keeps up to four 128-row tiles of the group's prompt queries resident in
+// shared memory (a tile packs two 64-row sub-blocks, possibly of two query heads); the key tiles stream past them
+// through a TMA ring, each read once per sweep.
 //
-//   kLse     CTA = 128 prompt rows of one query head (the stationary A operand); streams every 128-key tile of the
-//            unit as B.  D[row][key] lands in tensor memory with one prompt row per lane, so each thread keeps the
-//            online (max, sum exp2) of its own row without any cross-lane traffic  ->  row_stats, row_lse.
-//   kColsum  CTA = one 128-key tile (stationary A); streams every 128-row block of every query head of the group
-//            as B.  D[key][row]: one key per lane, so the sum over prompt rows of exp2(s - max) / sum is a private
-//            running sum per thread  ->  scores.
+//   kLse     D = Qtile x Ktile^T lands in tensor memory with one prompt row per lane, so each thread keeps the
+//            online (max, sum exp2) of its own rows without cross-lane traffic -> per-split partial row statistics.
+//   kColsum  D = Ktile x Qtile^T: one key per lane, so the sum over prompt rows of exp2(s - max) / sum is a private
+//            running sum per thread -> scores.  Its prologue merges the splits' partial statistics (fixed order).
 //
-// Warp roles (192 threads): warp 0 lane 0 issues TMA loads (128-byte swizzle) into a 4-stage shared-memory ring,
-// warp 1 owns tensor memory and its lane 0 issues tcgen05.mma (128 x 128 x 16, fp32 accumulate) into one of four
-// 128-column accumulators, warps 2-5 read accumulators back with tcgen05.ld and do the softmax arithmetic.
-// mbarriers connect the three; every wait is bounded and raises FINCH_DEV_TIMEOUT instead of hanging.
-// Candidate tiles never straddle the cache/chunk boundary: the cache's rows are tiled first, then the chunk's.
+// Warp roles (320 threads): warp 0 lane 0 issues TMA loads (128-byte swizzle), warp 1 owns tensor memory and its
+// lane 0 issues tcgen05.mma (128 x 128 x 16, fp32 accumulate), warps 2-9 form two softmax groups of four warps.
+// The groups take alternate key tiles and each has its own pair of 128-column accumulators, so no sum ever crosses
+// threads and every scheduler has two softmax warps to hide tcgen05.ld and MUFU latency.  mbarriers connect the
+// roles; every wait is bounded and raises FINCH_DEV_TIMEOUT instead of hanging.  Candidate tiles never straddle the cache/chunk
+// boundary: the cache's rows are tiled first, then the chunk's.
 #include <limits.h>
 
 #include "finch_internal.cuh"
@@ -24,23 +26,31 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kRows = 128;        // rows per operand tile = MMA M = MMA N
-constexpr int kStages = 4;        // shared-memory stages of the streamed operand
-constexpr int kAccBufs = 4;       // accumulators of 128 fp32 columns in tensor memory (4 x 128 = all 512 columns)
-constexpr int kTcThreads = 192;
-constexpr int kSlabBytes = kRows * 128;  // one 64-element (128-byte) wide slab of a 128-row tile
-constexpr int kAuxBytes = 1024 + 4 * 2 * kRows * 8;  // barriers, then per-warp double-buffered row statistics
+constexpr int kRows = 128;       // rows per operand tile = MMA M = MMA N
+constexpr int kSub = 64;         // prompt rows per sub-block (two per query tile)
+constexpr int kQTiles = 4;       // query tiles resident at a time
+constexpr int kGroups = 2;       // softmax groups (four warps each); group g takes the split's key tiles g, g+2, ..
+constexpr int kAccBufs = 4;      // accumulators of 128 fp32 columns in tensor memory (all 512 columns), two per group
+constexpr int kMaxStages = 4;    // key-tile ring
+constexpr int kTcThreads = 64 + kGroups * 128;
+constexpr int kSlabBytes = kRows * 128;                 // a 64-element (128-byte) wide slab of a 128-row tile
+constexpr int kStatsBytes = kGroups * 4 * kQTiles * kRows * 8;  // per softmax warp: (-max, 1/sum) of resident rows
+constexpr int kAuxBytes = 1024 + kStatsBytes;
+constexpr int kSmemLimit = 232448;                      // 227 KiB per CTA
 
 enum { kLse = 0, kColsum = 1 };
 
 struct TcParams {
     ModelView mv;
     BatchView bv;
-    float2 *row_stats;
-    float *row_lse;
+    float2 *partial;   // [splits][kGroups][L][Hq][total_q] (max base-2 logit, sum exp2) per prompt row and part
+    float *row_lse;    // nullable
     float *scores;
     int *status;
-    int min_q;  // requests with fewer prompt rows are left to the warp-level path
+    int min_q;         // requests with fewer prompt rows are left to the warp-level path
+    int splits;        // key splits per unit (grid x)
+    int stages;        // key-tile ring depth that fits beside the resident queries
+    int q_tiles;       // query tiles resident at a time (1..4), sized from the batch's longest prompt
 };
 
 struct KeyTile {
@@ -70,25 +80,101 @@ __device__ __forceinline__ KeyTile key_tile(const UnitInfo &u, int t) {
     return k;
 }
 
+// The group's prompt rows as a list of 64-row sub-blocks, head-major then position: sub-block sb covers rows
+// [p0, p0 + valid) of the group's query head hh.  Query tile t packs sub-blocks 2t and 2t + 1.
+struct SubBlock {
+    int hh, p0, valid;
+};
+__device__ __forceinline__ SubBlock sub_block(int sb, int sbq, int n_sb, int n_q) {
+    SubBlock s;
+    s.hh = sb / sbq;
+    s.p0 = (sb % sbq) * kSub;
+    s.valid = sb < n_sb ? min(kSub, n_q - s.p0) : 0;
+    return s;
+}
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// kLse: fold the first `valid` columns (keys) of one accumulator row into the row's online (max, sum).
+__device__ __forceinline__ void lse_accumulate(uint32_t taddr, int valid, float scale2, float &m_raw, float &z) {
+#pragma unroll 1
+    for (int cc = 0; cc * 32 < valid; ++cc) {
+        float v[32];
+        __syncwarp();
+        tmem_ld_x32(taddr + cc * 32, v);
+        const int nv = valid - cc * 32;
+        if (nv < 32) {
+#pragma unroll
+            for (int e = 1; e < 32; ++e) v[e] = e < nv ? v[e] : -INFINITY;  // columns past the last key count nothing
+        }
+        float cmax = v[0];
+#pragma unroll
+        for (int e = 1; e < 32; ++e) cmax = fmaxf(cmax, v[e]);
+        if (cmax > m_raw) {
+            z *= ex2((m_raw - cmax) * scale2);
+            m_raw = cmax;
+        }
+        const float negm = -(m_raw * scale2);
+        float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+            a0 += ex2(fmaf(v[e], scale2, negm));
+            a1 += ex2(fmaf(v[e + 1], scale2, negm));
+        }
+        z += a0 + a1;
+    }
+}
+
+// kColsum: add to (c0, c1) the weights exp2(s * scale2 - max_r) / sum_r of one accumulator row (a key) over the
+// valid prompt rows of the query tile: v0 rows in its first 64-row half, v1 in its second.  sm = (-max, 1/sum).
+__device__ __forceinline__ void colsum_accumulate(uint32_t taddr, int v0, int v1, float scale2, const float2 *sm,
+                                                  float &c0, float &c1) {
+    const float4 *sm4 = (const float4 *)sm;
+#pragma unroll 1
+    for (int cc = 0; cc < 4; ++cc) {
+        const int nv = min(32, (cc < 2 ? v0 : v1) - (cc & 1) * 32);
+        if (nv <= 0) continue;
+        float v[32];
+        __syncwarp();
+        tmem_ld_x32(taddr + cc * 32, v);
+        if (nv < 32) {
+#pragma unroll
+            for (int e = 1; e < 32; ++e) v[e] = e < nv ? v[e] : -INFINITY;  // rows past the prompt weigh nothing
+        }
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+            const float4 s4 = sm4[cc * 16 + e / 2];  // statistics of two prompt rows
+            c0 = fmaf(ex2(fmaf(v[e], scale2, s4.x)), s4.y, c0);
+            c1 = fmaf(ex2(fmaf(v[e + 1], scale2, s4.z)), s4.w, c1);
+        }
+    }
+}
+
 template <int MODE, int D>
 __global__ void __launch_bounds__(kTcThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap cache_map,
                 const __grid_constant__ CUtensorMap chunk_map, TcParams p) {
     constexpr int kSlabs = D / 64;
     constexpr int kTileBytes = kSlabs * kSlabBytes;
+    constexpr int kSubBytes = kSub * 128;  // the 64 rows of one sub-block inside one slab
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t *stat_tile = smem;
-    uint8_t *stage_tiles = smem + kTileBytes;
-    uint8_t *aux = stage_tiles + kStages * kTileBytes;
-    uint64_t *stat_full = (uint64_t *)aux;
-    uint64_t *full = stat_full + 1;
-    uint64_t *empty = full + kStages;
-    uint64_t *acc_full = empty + kStages;
+    uint8_t *q_res = smem;
+    uint8_t *k_ring = smem + p.q_tiles * kTileBytes;
+    uint8_t *aux = k_ring + p.stages * kTileBytes;
+    uint64_t *q_full = (uint64_t *)aux;
+    uint64_t *q_empty = q_full + 1;
+    uint64_t *full = q_empty + 1;
+    uint64_t *empty = full + kMaxStages;
+    uint64_t *acc_full = empty + kMaxStages;
     uint64_t *acc_empty = acc_full + kAccBufs;
     uint32_t *tmem_slot = (uint32_t *)(acc_empty + kAccBufs);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
-    float2 *stats_sm = (float2 *)(aux + 1024);  // [4 warps][2][128] (-max, 1/sum), kColsum only
+    float2 *stats_sm = (float2 *)(aux + 1024);  // [4 softmax warps][q_tiles * 128] (-max, 1/sum), kColsum only
 
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
@@ -99,28 +185,22 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     }
     if (u.n_q < p.min_q || u.N == 0) return;
     const int kvh = u.G;  // one KV head per selection group on this path
-    const int q_blocks = (u.n_q + kRows - 1) / kRows;
     const int k_tiles = n_key_tiles(u);
-
-    // ---- what this CTA holds still, and what it streams
-    int n_iter, hh_lse = 0, p0_lse = 0;
-    KeyTile my_tile{};
-    if (MODE == kLse) {
-        const int row_blocks = (bv.max_q + kRows - 1) / kRows;
-        hh_lse = blockIdx.x / row_blocks;
-        p0_lse = (blockIdx.x % row_blocks) * kRows;
-        if (p0_lse >= u.n_q) return;
-        n_iter = k_tiles;
-    } else {
-        if ((int)blockIdx.x >= k_tiles) return;
-        my_tile = key_tile(u, blockIdx.x);
-        n_iter = mv.hpg * q_blocks;
-    }
+    const int tps = (k_tiles + p.splits - 1) / p.splits;  // key tiles per split
+    const int split = blockIdx.x;
+    const int t0 = split * tps, t1 = min(k_tiles, t0 + tps);
+    if (t0 >= t1) return;
+    const int sbq = (u.n_q + kSub - 1) / kSub;  // sub-blocks per query head
+    const int n_sb = mv.hpg * sbq;
+    const int n_qt = (n_sb + 1) / 2;            // query tiles of the group
+    const int n_chunks = (n_qt + p.q_tiles - 1) / p.q_tiles;
+    const int64_t rows_total = (int64_t)mv.L * mv.Hq * bv.total_q;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        mbar_init(stat_full, 1);
-        for (int s = 0; s < kStages; ++s) {
+        mbar_init(q_full, 1);
+        mbar_init(q_empty, 1);
+        for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
         }
@@ -146,160 +226,177 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             prefetch_tensormap(&q_map);
             prefetch_tensormap(&cache_map);
             prefetch_tensormap(&chunk_map);
-            mbar_expect_tx(stat_full, kTileBytes);
-            if (MODE == kLse) {
-                const int h = u.G * mv.hpg + hh_lse;
-                for (int s = 0; s < kSlabs; ++s)
-                    tma_load_4d(stat_tile + s * kSlabBytes, &q_map, stat_full, s * 64, u.q0 + p0_lse, h, u.l);
-            } else {
-                const CUtensorMap *m = my_tile.is_chunk ? &chunk_map : &cache_map;
-                for (int s = 0; s < kSlabs; ++s)
-                    tma_load_4d(stat_tile + s * kSlabBytes, m, stat_full, s * 64, my_tile.row0, kvh, u.l);
-            }
-            int issued = 0;
-            for (int i = 0; i < n_iter; ++i) {
-                const int stage = i % kStages, ph = (i / kStages) & 1;
-                if (!mbar_wait(&empty[stage], ph ^ 1, abort_flag)) break;
-                mbar_expect_tx(&full[stage], kTileBytes);
-                uint8_t *dst = stage_tiles + stage * kTileBytes;
-                if (MODE == kLse) {
-                    const KeyTile kt = key_tile(u, i);
+            int kcnt = 0, q_issued = 0;
+            bool ok = true;
+            for (int c = 0; c < n_chunks && ok; ++c) {
+                const int qt0 = c * p.q_tiles;
+                const int nload = min(2 * min(p.q_tiles, n_qt - qt0), n_sb - 2 * qt0);
+                if (!mbar_wait(q_empty, (c & 1) ^ 1, abort_flag)) break;  // the previous chunk's MMAs have read it
+                mbar_expect_tx(q_full, nload * kSlabs * kSubBytes);
+                for (int sl = 0; sl < nload; ++sl) {
+                    const SubBlock sb = sub_block(2 * qt0 + sl, sbq, n_sb, u.n_q);
+                    uint8_t *dst = q_res + (sl / 2) * kTileBytes + (sl % 2) * kSubBytes;
+                    for (int s = 0; s < kSlabs; ++s)
+                        tma_load_4d(dst + s * kSlabBytes, &q_map, q_full, s * 64, u.q0 + sb.p0, u.G * mv.hpg + sb.hh, u.l);
+                }
+                ++q_issued;
+                for (int t = t0; t < t1; ++t, ++kcnt) {
+                    const int stage = kcnt % p.stages, ph = (kcnt / p.stages) & 1;
+                    if (!mbar_wait(&empty[stage], ph ^ 1, abort_flag)) { ok = false; break; }
+                    mbar_expect_tx(&full[stage], kTileBytes);
+                    const KeyTile kt = key_tile(u, t);
                     const CUtensorMap *m = kt.is_chunk ? &chunk_map : &cache_map;
                     for (int s = 0; s < kSlabs; ++s)
-                        tma_load_4d(dst + s * kSlabBytes, m, &full[stage], s * 64, kt.row0, kvh, u.l);
-                } else {
-                    const int h = u.G * mv.hpg + i / q_blocks, p0 = (i % q_blocks) * kRows;
-                    for (int s = 0; s < kSlabs; ++s)
-                        tma_load_4d(dst + s * kSlabBytes, &q_map, &full[stage], s * 64, u.q0 + p0, h, u.l);
+                        tma_load_4d(k_ring + stage * kTileBytes + s * kSlabBytes, m, &full[stage], s * 64, kt.row0, kvh,
+                                    u.l);
                 }
-                ++issued;
             }
-            // no copy may still be in flight when the CTA retires: wait (bounded) for the last ring of loads
-            mbar_wait(stat_full, 0, abort_flag);
-            for (int i = max(0, issued - kStages); i < issued; ++i)
-                mbar_wait(&full[i % kStages], (i / kStages) & 1, abort_flag);
+            // no copy may still be in flight when the CTA retires: wait (bounded) for the last loads issued
+            if (q_issued) mbar_wait(q_full, (q_issued - 1) & 1, abort_flag);
+            for (int i = max(0, kcnt - p.stages); i < kcnt; ++i)
+                mbar_wait(&full[i % p.stages], (i / p.stages) & 1, abort_flag);
         }
     } else if (warp == 1) {
         // =================================================================== MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_bf16_f32(kRows, kRows);
-            const uint32_t a_addr = smem_u32(stat_tile);
-            if (mbar_wait(stat_full, 0, abort_flag)) {
-                for (int i = 0; i < n_iter; ++i) {
-                    const int stage = i % kStages, ph = (i / kStages) & 1;
-                    const int buf = i % kAccBufs, bph = (i / kAccBufs) & 1;
-                    if (!mbar_wait(&full[stage], ph, abort_flag)) break;
-                    if (!mbar_wait(&acc_empty[buf], bph ^ 1, abort_flag)) break;
-                    tc_fence_after();
-                    const uint32_t b_addr = smem_u32(stage_tiles + stage * kTileBytes);
+            const uint32_t q_addr = smem_u32(q_res), ring_addr = smem_u32(k_ring);
+            int kcnt = 0, acnt[kGroups] = {0, 0};
+            bool ok = true;
+            for (int c = 0; c < n_chunks && ok; ++c) {
+                const int nqt = min(p.q_tiles, n_qt - c * p.q_tiles);
+                if (!mbar_wait(q_full, c & 1, abort_flag)) break;
+                for (int t = t0; t < t1 && ok; ++t, ++kcnt) {
+                    const int stage = kcnt % p.stages, ph = (kcnt / p.stages) & 1;
+                    const int g = (t - t0) & 1;  // softmax group that takes this key tile
+                    if (!mbar_wait(&full[stage], ph, abort_flag)) { ok = false; break; }
+                    for (int qb = 0; qb < nqt; ++qb, ++acnt[g]) {
+                        const int buf = 2 * g + (acnt[g] & 1), bph = (acnt[g] >> 1) & 1;
+                        if (!mbar_wait(&acc_empty[buf], bph ^ 1, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t qa = q_addr + qb * kTileBytes, ka = ring_addr + stage * kTileBytes;
+                        const uint32_t a_addr = MODE == kLse ? qa : ka, b_addr = MODE == kLse ? ka : qa;
 #pragma unroll
-                    for (int k = 0; k < D / 16; ++k) {
-                        const uint32_t off = (k / 4) * kSlabBytes + (k % 4) * 32;
-                        umma_bf16(tmem_base + buf * kRows, smem_desc_sw128(a_addr + off), smem_desc_sw128(b_addr + off),
-                                  idesc, k > 0);
+                        for (int k = 0; k < D / 16; ++k) {
+                            const uint32_t off = (k / 4) * kSlabBytes + (k % 4) * 32;
+                            umma_bf16(tmem_base + buf * kRows, smem_desc_sw128(a_addr + off),
+                                      smem_desc_sw128(b_addr + off), idesc, k > 0);
+                        }
+                        umma_commit(&acc_full[buf]);  // the accumulator is ready for its softmax group
                     }
-                    umma_commit(&empty[stage]);   // the stage may be refilled once these MMAs have read it
-                    umma_commit(&acc_full[buf]);  // and the accumulator is ready for the softmax warps
+                    if (ok) umma_commit(&empty[stage]);  // the stage may be refilled once these MMAs have read it
                 }
+                if (ok) umma_commit(q_empty);
             }
         }
     } else {
         // =================================================================== softmax warps (one TMEM lane per thread)
-        const int quarter = warp & 3;                       // tcgen05.ld reaches lanes 32*(warp % 4) ..
-        const int my_row = quarter * 32 + lane;             // row of the stationary tile this thread owns
+        const int quarter = warp & 3;            // tcgen05.ld reaches lanes 32 * (warp % 4) ..
+        const int g = (warp - 2) >> 2;           // softmax group: key tiles t0 + g, t0 + g + 2, ..
+        const int my_row = quarter * 32 + lane;  // row of the A tile this thread owns
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
         const float scale2 = mv.scale * kLog2e;
-        float v[32];
-        if (MODE == kLse) {
-            float m_raw = -INFINITY, z = 0.f;
-            bool done = true;
-            for (int i = 0; i < n_iter; ++i) {
-                const int buf = i % kAccBufs, bph = (i / kAccBufs) & 1;
-                const KeyTile kt = key_tile(u, i);
-                // the verdict of a wait is made warp-uniform so that a timeout takes the whole warp out of the loop
-                if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[buf], bph, abort_flag))) { done = false; break; }
-                tc_fence_after();
-                for (int cc = 0; cc * 32 < kt.valid; ++cc) {
-                    __syncwarp();
-                    tmem_ld_x32(t_lane + buf * kRows + cc * 32, v);
-                    const int nv = kt.valid - cc * 32;
-                    float cmax = v[0];
-                    if (nv >= 32) {
+        int acnt = 0;
+        bool ok = true;
+        for (int c = 0; c < n_chunks && ok; ++c) {
+            const int qt0 = c * p.q_tiles;
+            const int nqt = min(p.q_tiles, n_qt - qt0);
+            if (MODE == kLse) {
+                float m_raw[kQTiles], z[kQTiles];
 #pragma unroll
-                        for (int e = 1; e < 32; ++e) cmax = fmaxf(cmax, v[e]);
-                    } else {
+                for (int k = 0; k < kQTiles; ++k) {
+                    m_raw[k] = -INFINITY;
+                    z[k] = 0.f;
+                }
+                for (int t = t0 + g; t < t1 && ok; t += kGroups) {
+                    const KeyTile kt = key_tile(u, t);
+#pragma unroll 1
+                    for (int qb = 0; qb < nqt && ok; ++qb, ++acnt) {
+                        const int buf = 2 * g + (acnt & 1), bph = (acnt >> 1) & 1;
+                        // a wait's verdict is made warp-uniform so that a timeout takes the whole warp out
+                        if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[buf], bph, abort_flag))) { ok = false; break; }
+                        tc_fence_after();
+                        float mc = 0.f, zc = 0.f;  // the running statistics of query tile qb (kept in registers)
 #pragma unroll
-                        for (int e = 1; e < 32; ++e) cmax = e < nv ? fmaxf(cmax, v[e]) : cmax;
-                    }
-                    if (cmax > m_raw) {
-                        z *= exp2f((m_raw - cmax) * scale2);
-                        m_raw = cmax;
-                    }
-                    const float negm = -(m_raw * scale2);
-                    if (nv >= 32) {
+                        for (int k = 0; k < kQTiles; ++k)
+                            if (k == qb) {
+                                mc = m_raw[k];
+                                zc = z[k];
+                            }
+                        lse_accumulate(t_lane + buf * kRows, kt.valid, scale2, mc, zc);
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) z += exp2f(fmaf(v[e], scale2, negm));
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) z += e < nv ? exp2f(fmaf(v[e], scale2, negm)) : 0.f;
+                        for (int k = 0; k < kQTiles; ++k)
+                            if (k == qb) {
+                                m_raw[k] = mc;
+                                z[k] = zc;
+                            }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&acc_empty[buf]);
                     }
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&acc_empty[buf]);
-            }
-            const int prow = p0_lse + my_row;
-            if (done && prow < u.n_q) {
-                const int h = u.G * mv.hpg + hh_lse;
-                const int64_t row = ((int64_t)u.l * mv.Hq + h) * bv.total_q + u.q0 + prow;
-                const float m2 = m_raw * scale2;
-                p.row_stats[row] = make_float2(m2, 1.0f / z);
-                if (p.row_lse) p.row_lse[row] = (m2 + log2f(z)) * kLn2;
-            }
-        } else {
-            float col = 0.f;
-            bool done = true;
-            for (int i = 0; i < n_iter; ++i) {
-                const int buf = i % kAccBufs, bph = (i / kAccBufs) & 1;
-                const int h = u.G * mv.hpg + i / q_blocks, p0 = (i % q_blocks) * kRows;
-                const int nvalid = min(kRows, u.n_q - p0);
-                // each warp stages the row block's statistics for itself (no CTA-wide barrier inside this loop)
-                float2 *sm = stats_sm + ((warp - 2) * 2 + (i & 1)) * kRows;
-                const float2 *gstats = p.row_stats + ((int64_t)u.l * mv.Hq + h) * bv.total_q + u.q0 + p0;
-                for (int t = lane; t < kRows; t += 32) {
-                    const float2 st = t < nvalid ? gstats[t] : make_float2(0.f, 0.f);
-                    sm[t] = make_float2(-st.x, st.y);
-                }
-                __syncwarp();
-                if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[buf], bph, abort_flag))) { done = false; break; }
-                tc_fence_after();
-                for (int cc = 0; cc * 32 < nvalid; ++cc) {
-                    __syncwarp();
-                    tmem_ld_x32(t_lane + buf * kRows + cc * 32, v);
-                    const int nv = nvalid - cc * 32;
-                    if (nv >= 32) {
+                if (ok && t0 + g < t1) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) {
-                            const float2 s2 = sm[cc * 32 + e];
-                            col = fmaf(exp2f(fmaf(v[e], scale2, s2.x)), s2.y, col);
+                    for (int qb = 0; qb < kQTiles; ++qb) {
+                        if (qb >= nqt) continue;
+                        const SubBlock sb = sub_block(2 * (qt0 + qb) + my_row / kSub, sbq, n_sb, u.n_q);
+                        const int r = my_row % kSub;
+                        if (r < sb.valid) {
+                            const int64_t row = ((int64_t)u.l * mv.Hq + u.G * mv.hpg + sb.hh) * bv.total_q + u.q0 + sb.p0 + r;
+                            p.partial[(split * kGroups + g) * rows_total + row] = make_float2(m_raw[qb] * scale2, z[qb]);
                         }
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) {
-                            if (e < nv) {
-                                const float2 s2 = sm[cc * 32 + e];
-                                col = fmaf(exp2f(fmaf(v[e], scale2, s2.x)), s2.y, col);
+                    }
+                }
+            } else {
+                // merge the partial statistics of this chunk's rows (every key split, both groups), each warp for
+                // itself and all in the same order, so that every CTA of the unit uses identical values
+                float2 *sm = stats_sm + (warp - 2) * kQTiles * kRows;
+                for (int idx = lane; idx < nqt * kRows; idx += 32) {
+                    const int r = idx % kRows;
+                    const SubBlock sb = sub_block(2 * (qt0 + idx / kRows) + r / kSub, sbq, n_sb, u.n_q);
+                    float2 out = make_float2(0.f, 0.f);
+                    if (r % kSub < sb.valid) {
+                        const int64_t row = ((int64_t)u.l * mv.Hq + u.G * mv.hpg + sb.hh) * bv.total_q + u.q0 + sb.p0 +
+                                            r % kSub;
+                        float M = -INFINITY, Z = 0.f;
+                        for (int s = 0; s * tps < k_tiles; ++s) {
+                            const int parts = min(kGroups, min(k_tiles, (s + 1) * tps) - s * tps);
+                            for (int gg = 0; gg < parts; ++gg) {
+                                const float2 pm = p.partial[(s * kGroups + gg) * rows_total + row];
+                                const float nm = fmaxf(M, pm.x);
+                                Z = Z * ex2(M - nm) + pm.y * ex2(pm.x - nm);
+                                M = nm;
                             }
                         }
+                        out = make_float2(-M, 1.0f / Z);
+                        if (split == 0 && warp == 2 && p.row_lse) p.row_lse[row] = (M + log2f(Z)) * kLn2;
+                    }
+                    sm[idx] = out;
+                }
+                __syncwarp();
+                for (int t = t0 + g; t < t1 && ok; t += kGroups) {
+                    const KeyTile kt = key_tile(u, t);
+                    float c0 = 0.f, c1 = 0.f;
+#pragma unroll 1
+                    for (int qb = 0; qb < nqt && ok; ++qb, ++acnt) {
+                        const int buf = 2 * g + (acnt & 1), bph = (acnt >> 1) & 1;
+                        if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[buf], bph, abort_flag))) { ok = false; break; }
+                        tc_fence_after();
+                        const int v0 = sub_block(2 * (qt0 + qb), sbq, n_sb, u.n_q).valid;
+                        const int v1 = sub_block(2 * (qt0 + qb) + 1, sbq, n_sb, u.n_q).valid;
+                        colsum_accumulate(t_lane + buf * kRows, v0, v1, scale2, sm + qb * kRows, c0, c1);
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                    }
+                    if (ok && my_row < kt.valid) {
+                        float *dst = p.scores + ((int64_t)u.l * mv.G + u.G) * ((int64_t)bv.total_cache + bv.total_chunk) +
+                                     u.cache0 + u.chunk0 + kt.j0 + my_row;
+                        const float col = c0 + c1;
+                        *dst = c == 0 ? col : *dst + col;  // later query chunks add to the first chunk's sums
                     }
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&acc_empty[buf]);
             }
-            if (done && my_row < my_tile.valid)
-                p.scores[((int64_t)u.l * mv.G + u.G) * ((int64_t)bv.total_cache + bv.total_chunk) + u.cache0 + u.chunk0 +
-                         my_tile.j0 + my_row] = col;
         }
     }
 
@@ -334,8 +431,8 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// [layers][heads][tokens][d] bf16 view -> 4-D tensor map with a (64 elements x 128 rows) box, 128-byte swizzle.
-bool make_map(CUtensorMap *map, const TensorView &t, int d, int64_t tokens, int heads, int layers) {
+// [layers][heads][tokens][d] bf16 view -> 4-D tensor map with a (64 elements x box_rows) box, 128-byte swizzle.
+bool make_map(CUtensorMap *map, const TensorView &t, int d, int64_t tokens, int heads, int layers, int box_rows) {
     EncodeTiledFn fn = encode_fn();
     if (!fn || !t.ptr || tokens <= 0) return false;
     const cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)tokens, (cuuint64_t)heads, (cuuint64_t)layers};
@@ -343,30 +440,47 @@ bool make_map(CUtensorMap *map, const TensorView &t, int d, int64_t tokens, int 
                                    (cuuint64_t)t.stride_layer * 2};
     for (int i = 0; i < 3; ++i)
         if (strides[i] == 0 || strides[i] % 16 || strides[i] >= (1ull << 40)) return false;
-    const cuuint32_t box[4] = {64, (cuuint32_t)kRows, 1, 1};
+    const cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<char *>(t.ptr), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Key splits per unit: the smallest count (at most max_splits, at least one key tile each) whose grid fills whole
+// waves of SMs best.
+int choose_splits(int ctas_per_split, int key_tiles, int sm_count, int max_splits) {
+    int best = 1;
+    double best_eff = 0.0;
+    for (int s = 1; s <= max_splits && s <= key_tiles; ++s) {
+        const double waves = (double)ctas_per_split * s / sm_count;
+        const double eff = waves / (double)((long long)waves + (waves > (long long)waves ? 1 : 0));
+        if (eff > best_eff * 1.05) {
+            best_eff = eff;
+            best = s;
+        }
+    }
+    return best;
+}
+
 template <int D>
-cudaError_t launch_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensorMap &cm, const CUtensorMap &hm,
-                     const TcParams &p, cudaStream_t stream) {
-    constexpr int kSmem = 1024 + (1 + kStages) * (D / 64) * kSlabBytes + kAuxBytes;
+cudaError_t launch_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensorMap &cm, const CUtensorMap &hm, TcParams p,
+                     cudaStream_t stream) {
+    constexpr int kTileBytes = (D / 64) * kSlabBytes;
     const ModelView &mv = ctx.model;
     const BatchView &bv = p.bv;
-    cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<kLse, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    const int sub_blocks = mv.hpg * ((bv.max_q + kSub - 1) / kSub);
+    p.q_tiles = min(kQTiles, (sub_blocks + 1) / 2);
+    p.stages = min(kMaxStages, (kSmemLimit - 1024 - kAuxBytes - p.q_tiles * kTileBytes) / kTileBytes);
+    if (p.stages < 2) return cudaErrorNotSupported;
+    const int smem = 1024 + (p.q_tiles + p.stages) * kTileBytes + kAuxBytes;
+    cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<kLse, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(score_tc_kernel<kColsum, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    e = cudaFuncSetAttribute(score_tc_kernel<kColsum, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    const int units = mv.L * mv.G;
-    const int row_blocks = (bv.max_q + kRows - 1) / kRows;
-    const int key_tiles = (bv.max_cache + kRows - 1) / kRows + (bv.max_chunk + kRows - 1) / kRows;
-    dim3 g1(row_blocks * mv.hpg, units, bv.batch);
-    score_tc_kernel<kLse, D><<<g1, kTcThreads, kSmem, stream>>>(qm, cm, hm, p);
-    dim3 g2(key_tiles, units, bv.batch);
-    score_tc_kernel<kColsum, D><<<g2, kTcThreads, kSmem, stream>>>(qm, cm, hm, p);
+    dim3 grid(p.splits, mv.L * mv.G, bv.batch);
+    score_tc_kernel<kLse, D><<<grid, kTcThreads, smem, stream>>>(qm, cm, hm, p);
+    score_tc_kernel<kColsum, D><<<grid, kTcThreads, smem, stream>>>(qm, cm, hm, p);
     ctx.launches += 2;
     return cudaGetLastError();
 }
@@ -377,21 +491,27 @@ bool score_tc_supported(const Ctx &ctx) {
     return ctx.cfg.dtype == FINCH_BF16 && (ctx.model.d == 64 || ctx.model.d == 128) && ctx.model.kvpg == 1;
 }
 
-// Returns cudaErrorNotSupported (and launches nothing) when the tensors cannot be described to the TMA unit; the
-// caller then uses the warp-level path for every request.
+// `partial` holds partial_capacity float2 entries; the key-split count is limited so that one entry per prompt
+// row, split and softmax group fits.  Returns cudaErrorNotSupported (and launches nothing) when the tensors cannot be described
+// to the TMA unit; the caller then uses the warp-level path for every request.
 cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
-                            const BatchView &bv, float *scores, float2 *row_stats, float *row_lse, int min_q,
-                            cudaStream_t stream) {
+                            const BatchView &bv, float *scores, float2 *partial, size_t partial_capacity,
+                            float *row_lse, int min_q, cudaStream_t stream) {
     const ModelView &mv = ctx.model;
     if (mv.L * mv.G == 0 || bv.batch == 0 || bv.max_q == 0 || bv.max_cache + bv.max_chunk == 0) return cudaSuccess;
+    const size_t rows = (size_t)mv.L * mv.Hq * (size_t)bv.total_q;
+    if (rows == 0 || partial_capacity < rows * kGroups) return cudaErrorNotSupported;
     CUtensorMap qm, cm, hm;
-    if (!make_map(&qm, q, mv.d, bv.total_q, mv.Hq, mv.L)) return cudaErrorNotSupported;
+    if (!make_map(&qm, q, mv.d, bv.total_q, mv.Hq, mv.L, kSub)) return cudaErrorNotSupported;
     const bool have_cache = bv.max_cache > 0, have_chunk = bv.max_chunk > 0;
-    if (have_cache && !make_map(&cm, cache_k, mv.d, bv.total_cache, mv.Hkv, mv.L)) return cudaErrorNotSupported;
-    if (have_chunk && !make_map(&hm, chunk_k, mv.d, bv.total_chunk, mv.Hkv, mv.L)) return cudaErrorNotSupported;
+    if (have_cache && !make_map(&cm, cache_k, mv.d, bv.total_cache, mv.Hkv, mv.L, kRows)) return cudaErrorNotSupported;
+    if (have_chunk && !make_map(&hm, chunk_k, mv.d, bv.total_chunk, mv.Hkv, mv.L, kRows)) return cudaErrorNotSupported;
     if (!have_cache) cm = hm;  // never dereferenced: no request has cache tiles
     if (!have_chunk) hm = cm;
-    TcParams p{mv, bv, row_stats, row_lse, scores, ctx.d_status, min_q};
+    const int key_tiles = (bv.max_cache + kRows - 1) / kRows + (bv.max_chunk + kRows - 1) / kRows;
+    const int max_splits = (int)min((size_t)kScoreMaxSplits, partial_capacity / (rows * kGroups));
+    TcParams p{mv, bv, partial, row_lse, scores, ctx.d_status, min_q, 1, 2, 1};
+    p.splits = choose_splits(mv.L * mv.G * bv.batch, key_tiles, ctx.sm_count > 0 ? ctx.sm_count : 148, max_splits);
     return mv.d == 64 ? launch_d<64>(ctx, qm, cm, hm, p, stream) : launch_d<128>(ctx, qm, cm, hm, p, stream);
 }
 
