@@ -43,7 +43,8 @@ enum { kLse = 0, kColsum = 1 };
 struct TcParams {
     ModelView mv;
     BatchView bv;
-    float2 *partial;   // [splits][kGroups][L][Hq][total_q] (max base-2 logit, sum exp2) per prompt row and part
+    float2 *partial;   // [splits][kGroups][L][Hq][total_q] (reference base-2 logit, sum exp2) per prompt row and part
+    float2 *merged;    // [L][Hq][total_q] (-reference, weight) per prompt row after merging the parts
     float *row_lse;    // nullable
     float *scores;
     int *status;
@@ -99,25 +100,26 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
-// kLse: fold the first `valid` columns (keys) of one accumulator row into the row's online (max, sum).
-__device__ __forceinline__ void lse_accumulate(uint32_t taddr, int valid, float scale2, float &m_raw, float &z) {
-#pragma unroll 1
-    for (int cc = 0; cc * 32 < valid; ++cc) {
-        float v[32];
-        __syncwarp();
-        tmem_ld_x32(taddr + cc * 32, v);
-        const int nv = valid - cc * 32;
-        if (nv < 32) {
+// kLse: fold 32 columns (keys) of one accumulator row into the row's running (reference, sum of exp2).
+// The reference is the maximum of the row's first chunk, not the running maximum: any reference works as long as
+// the sum stays finite, and skipping the per-element maximum saves a quarter of the instructions.  If the sum
+// overflows (a later logit more than ~2^7 base-2 units above the reference) the reference is raised and the chunk
+// redone.  Columns at or beyond nv hold no key and count nothing.
+__device__ __forceinline__ void lse_chunk(const uint32_t (&r)[32], int nv, float scale2, float &m_raw, float &z) {
+    float v[32];
 #pragma unroll
-            for (int e = 1; e < 32; ++e) v[e] = e < nv ? v[e] : -INFINITY;  // columns past the last key count nothing
-        }
+    for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]);
+    if (nv < 32) {
+#pragma unroll
+        for (int e = 1; e < 32; ++e) v[e] = e < nv ? v[e] : -INFINITY;
+    }
+    if (m_raw == -INFINITY) {
         float cmax = v[0];
 #pragma unroll
         for (int e = 1; e < 32; ++e) cmax = fmaxf(cmax, v[e]);
-        if (cmax > m_raw) {
-            z *= ex2((m_raw - cmax) * scale2);
-            m_raw = cmax;
-        }
+        m_raw = cmax;
+    }
+    for (int attempt = 0; attempt < 8; ++attempt) {
         const float negm = -(m_raw * scale2);
         float a0 = 0.f, a1 = 0.f;
 #pragma unroll
@@ -125,32 +127,71 @@ __device__ __forceinline__ void lse_accumulate(uint32_t taddr, int valid, float 
             a0 += ex2(fmaf(v[e], scale2, negm));
             a1 += ex2(fmaf(v[e + 1], scale2, negm));
         }
-        z += a0 + a1;
+        const float zn = z + (a0 + a1);
+        if (!(zn > 3.0e38f)) {  // finite -- or NaN, on a lane that holds no prompt row: nothing to repair
+            z = zn;
+            break;
+        }
+        m_raw += 64.0f / scale2;  // overflow: lift the reference by 2^64 and rescale what has been summed so far
+        z *= 5.421010862427522e-20f;
     }
 }
 
-// kColsum: add to (c0, c1) the weights exp2(s * scale2 - max_r) / sum_r of one accumulator row (a key) over the
-// valid prompt rows of the query tile: v0 rows in its first 64-row half, v1 in its second.  sm = (-max, 1/sum).
+// `live` is false on lanes whose row of the query tile holds no prompt row: they take part in the (warp-wide)
+// loads but skip the arithmetic, whose input would be whatever the shared memory held before.
+__device__ __forceinline__ void lse_accumulate(uint32_t taddr, int valid, float scale2, bool live, float &m_raw,
+                                               float &z) {
+    uint32_t r[2][32];
+    __syncwarp();
+    tmem_ld_x32_issue(taddr, r[0]);
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc) {
+        if (cc * 32 >= valid) break;
+        tmem_ld_x32_wait(r[cc & 1]);
+        if ((cc + 1) * 32 < valid) {  // start the next chunk's load before working on this one
+            __syncwarp();
+            tmem_ld_x32_issue(taddr + (cc + 1) * 32, r[(cc + 1) & 1]);
+        }
+        if (live) lse_chunk(r[cc & 1], valid - cc * 32, scale2, m_raw, z);
+    }
+}
+
+// kColsum: add to (c0, c1) the weights exp2(s * scale2 - ref_r) * w_r of one accumulator row (a key) over the valid
+// prompt rows of the query tile: v0 rows in its first 64-row half, v1 in its second.  sm[r] = (-ref_r, w_r).
+__device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[32], int nv, float scale2, const float4 *sm4, float &c0,
+                                             float &c1) {
+    float v[32];
+#pragma unroll
+    for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]);
+    if (nv < 32) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) v[e] = e < nv ? v[e] : -INFINITY;  // rows past the prompt weigh nothing
+    }
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) {
+        const float4 s4 = sm4[e / 2];  // statistics of two prompt rows
+        c0 = fmaf(ex2(fmaf(v[e], scale2, s4.x)), s4.y, c0);
+        c1 = fmaf(ex2(fmaf(v[e + 1], scale2, s4.z)), s4.w, c1);
+    }
+}
+
 __device__ __forceinline__ void colsum_accumulate(uint32_t taddr, int v0, int v1, float scale2, const float2 *sm,
                                                   float &c0, float &c1) {
     const float4 *sm4 = (const float4 *)sm;
-#pragma unroll 1
+    uint32_t r[2][32];
+    // chunks 0 and 1 cover the tile's first 64-row half (always present), chunks 2 and 3 the second half
+    const int last = v1 > 0 ? 4 : 2;
+    __syncwarp();
+    tmem_ld_x32_issue(taddr, r[0]);
+#pragma unroll
     for (int cc = 0; cc < 4; ++cc) {
-        const int nv = min(32, (cc < 2 ? v0 : v1) - (cc & 1) * 32);
-        if (nv <= 0) continue;
-        float v[32];
-        __syncwarp();
-        tmem_ld_x32(taddr + cc * 32, v);
-        if (nv < 32) {
-#pragma unroll
-            for (int e = 1; e < 32; ++e) v[e] = e < nv ? v[e] : -INFINITY;  // rows past the prompt weigh nothing
+        if (cc >= last) break;
+        tmem_ld_x32_wait(r[cc & 1]);
+        if (cc + 1 < last) {  // start the next chunk's load before working on this one
+            __syncwarp();
+            tmem_ld_x32_issue(taddr + (cc + 1) * 32, r[(cc + 1) & 1]);
         }
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-            const float4 s4 = sm4[cc * 16 + e / 2];  // statistics of two prompt rows
-            c0 = fmaf(ex2(fmaf(v[e], scale2, s4.x)), s4.y, c0);
-            c1 = fmaf(ex2(fmaf(v[e + 1], scale2, s4.z)), s4.w, c1);
-        }
+        colsum_chunk(r[cc & 1], (cc < 2 ? v0 : v1) - (cc & 1) * 32, scale2, sm4 + cc * 16, c0, c1);
     }
 }
 
@@ -303,10 +344,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             const int nqt = min(p.q_tiles, n_qt - qt0);
             if (MODE == kLse) {
                 float m_raw[kQTiles], z[kQTiles];
+                uint32_t live_mask = 0;  // bit qb: this thread's row of query tile qb holds a prompt row
 #pragma unroll
                 for (int k = 0; k < kQTiles; ++k) {
                     m_raw[k] = -INFINITY;
                     z[k] = 0.f;
+                    if (k < nqt && my_row % kSub < sub_block(2 * (qt0 + k) + my_row / kSub, sbq, n_sb, u.n_q).valid)
+                        live_mask |= 1u << k;
                 }
                 for (int t = t0 + g; t < t1 && ok; t += kGroups) {
                     const KeyTile kt = key_tile(u, t);
@@ -323,7 +367,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                                 mc = m_raw[k];
                                 zc = z[k];
                             }
-                        lse_accumulate(t_lane + buf * kRows, kt.valid, scale2, mc, zc);
+                        lse_accumulate(t_lane + buf * kRows, kt.valid, scale2, (live_mask >> qb) & 1u, mc, zc);
 #pragma unroll
                         for (int k = 0; k < kQTiles; ++k)
                             if (k == qb) {
@@ -348,29 +392,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                     }
                 }
             } else {
-                // merge the partial statistics of this chunk's rows (every key split, both groups), each warp for
-                // itself and all in the same order, so that every CTA of the unit uses identical values
+                // stage the merged statistics of this chunk's rows, each warp for itself
                 float2 *sm = stats_sm + (warp - 2) * kQTiles * kRows;
                 for (int idx = lane; idx < nqt * kRows; idx += 32) {
                     const int r = idx % kRows;
                     const SubBlock sb = sub_block(2 * (qt0 + idx / kRows) + r / kSub, sbq, n_sb, u.n_q);
                     float2 out = make_float2(0.f, 0.f);
-                    if (r % kSub < sb.valid) {
-                        const int64_t row = ((int64_t)u.l * mv.Hq + u.G * mv.hpg + sb.hh) * bv.total_q + u.q0 + sb.p0 +
-                                            r % kSub;
-                        float M = -INFINITY, Z = 0.f;
-                        for (int s = 0; s * tps < k_tiles; ++s) {
-                            const int parts = min(kGroups, min(k_tiles, (s + 1) * tps) - s * tps);
-                            for (int gg = 0; gg < parts; ++gg) {
-                                const float2 pm = p.partial[(s * kGroups + gg) * rows_total + row];
-                                const float nm = fmaxf(M, pm.x);
-                                Z = Z * ex2(M - nm) + pm.y * ex2(pm.x - nm);
-                                M = nm;
-                            }
-                        }
-                        out = make_float2(-M, 1.0f / Z);
-                        if (split == 0 && warp == 2 && p.row_lse) p.row_lse[row] = (M + log2f(Z)) * kLn2;
-                    }
+                    if (r % kSub < sb.valid)
+                        out = p.merged[((int64_t)u.l * mv.Hq + u.G * mv.hpg + sb.hh) * bv.total_q + u.q0 + sb.p0 + r % kSub];
                     sm[idx] = out;
                 }
                 __syncwarp();
@@ -409,6 +438,37 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         tc_fence_after();
         tmem_dealloc(tmem_base, 512);
     }
+}
+
+// Merge the per-split, per-group partial statistics of every prompt row (fixed order) into the pair the column pass
+// uses: weights are exp2(s2 - R) * w with R = M + floor(log2 Z) and w = 2^floor(log2 Z) / Z in (1/2, 1], so the
+// exponent never exceeds a few units whatever reference the parts were summed against.
+__global__ void __launch_bounds__(128)
+merge_stats_kernel(TcParams p) {
+    const ModelView &mv = p.mv;
+    const BatchView &bv = p.bv;
+    const int h = blockIdx.y % mv.Hq, l = blockIdx.y / mv.Hq;
+    const UnitInfo u = unit_info(mv, bv, l * mv.G + h / mv.hpg, blockIdx.z);
+    if (!u.ok || u.n_q < p.min_q || u.N == 0) return;
+    const int pr = blockIdx.x * 128 + threadIdx.x;
+    if (pr >= u.n_q) return;
+    const int k_tiles = n_key_tiles(u);
+    const int tps = (k_tiles + p.splits - 1) / p.splits;
+    const int64_t rows_total = (int64_t)mv.L * mv.Hq * bv.total_q;
+    const int64_t row = ((int64_t)l * mv.Hq + h) * bv.total_q + u.q0 + pr;
+    float M = -INFINITY, Z = 0.f;
+    for (int s = 0; s * tps < k_tiles; ++s) {
+        const int parts = min(kGroups, min(k_tiles, (s + 1) * tps) - s * tps);
+        for (int g = 0; g < parts; ++g) {
+            const float2 pm = p.partial[(s * kGroups + g) * rows_total + row];
+            const float nm = fmaxf(M, pm.x);
+            Z = Z * ex2(M - nm) + pm.y * ex2(pm.x - nm);
+            M = nm;
+        }
+    }
+    const int k = ilogbf(Z);
+    p.merged[row] = make_float2(-(M + (float)k), ldexpf(1.0f, k) / Z);
+    if (p.row_lse) p.row_lse[row] = (M + log2f(Z)) * kLn2;
 }
 
 // ------------------------------------------------------------------------------------------------ host side
@@ -480,8 +540,10 @@ cudaError_t launch_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensorMap &c
     if (e != cudaSuccess) return e;
     dim3 grid(p.splits, mv.L * mv.G, bv.batch);
     score_tc_kernel<kLse, D><<<grid, kTcThreads, smem, stream>>>(qm, cm, hm, p);
+    dim3 mgrid((bv.max_q + 127) / 128, mv.L * mv.Hq, bv.batch);
+    merge_stats_kernel<<<mgrid, 128, 0, stream>>>(p);
     score_tc_kernel<kColsum, D><<<grid, kTcThreads, smem, stream>>>(qm, cm, hm, p);
-    ctx.launches += 2;
+    ctx.launches += 3;
     return cudaGetLastError();
 }
 
@@ -492,7 +554,7 @@ bool score_tc_supported(const Ctx &ctx) {
 }
 
 // `partial` holds partial_capacity float2 entries; the key-split count is limited so that one entry per prompt
-// row, split and softmax group fits.  Returns cudaErrorNotSupported (and launches nothing) when the tensors cannot be described
+// row, split and softmax group, plus one merged entry per row, fits.  Returns cudaErrorNotSupported (and launches nothing) when the tensors cannot be described
 // to the TMA unit; the caller then uses the warp-level path for every request.
 cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
                             const BatchView &bv, float *scores, float2 *partial, size_t partial_capacity,
@@ -500,7 +562,7 @@ cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorVie
     const ModelView &mv = ctx.model;
     if (mv.L * mv.G == 0 || bv.batch == 0 || bv.max_q == 0 || bv.max_cache + bv.max_chunk == 0) return cudaSuccess;
     const size_t rows = (size_t)mv.L * mv.Hq * (size_t)bv.total_q;
-    if (rows == 0 || partial_capacity < rows * kGroups) return cudaErrorNotSupported;
+    if (rows == 0 || partial_capacity < rows * (kGroups + 1)) return cudaErrorNotSupported;
     CUtensorMap qm, cm, hm;
     if (!make_map(&qm, q, mv.d, bv.total_q, mv.Hq, mv.L, kSub)) return cudaErrorNotSupported;
     const bool have_cache = bv.max_cache > 0, have_chunk = bv.max_chunk > 0;
@@ -509,9 +571,10 @@ cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorVie
     if (!have_cache) cm = hm;  // never dereferenced: no request has cache tiles
     if (!have_chunk) hm = cm;
     const int key_tiles = (bv.max_cache + kRows - 1) / kRows + (bv.max_chunk + kRows - 1) / kRows;
-    const int max_splits = (int)min((size_t)kScoreMaxSplits, partial_capacity / (rows * kGroups));
-    TcParams p{mv, bv, partial, row_lse, scores, ctx.d_status, min_q, 1, 2, 1};
+    const int max_splits = (int)min((size_t)kScoreMaxSplits, (partial_capacity / rows - 1) / kGroups);
+    TcParams p{mv, bv, partial, nullptr, row_lse, scores, ctx.d_status, min_q, 1, 2, 1};
     p.splits = choose_splits(mv.L * mv.G * bv.batch, key_tiles, ctx.sm_count > 0 ? ctx.sm_count : 148, max_splits);
+    p.merged = partial + (size_t)p.splits * kGroups * rows;
     return mv.d == 64 ? launch_d<64>(ctx, qm, cm, hm, p, stream) : launch_d<128>(ctx, qm, cm, hm, p, stream);
 }
 
