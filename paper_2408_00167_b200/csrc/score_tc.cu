@@ -302,20 +302,29 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_bf16_f32(kRows, kRows);
             const uint32_t q_addr = smem_u32(q_res), ring_addr = smem_u32(k_ring);
-            int kcnt = 0, acnt[kGroups] = {0, 0};
+            // The two softmax groups consume independent streams of accumulators (group g: key tiles t0 + g,
+            // t0 + g + 2, .. of the split, every resident query tile of each).  The issuer serves whichever group
+            // has a free accumulator and a loaded key tile, so neither group waits for the other's backlog.
+            const int n_t = t1 - t0;
             bool ok = true;
+            int acnt[kGroups] = {0, 0};
             for (int c = 0; c < n_chunks && ok; ++c) {
                 const int nqt = min(p.q_tiles, n_qt - c * p.q_tiles);
                 if (!mbar_wait(q_full, c & 1, abort_flag)) break;
-                for (int t = t0; t < t1 && ok; ++t, ++kcnt) {
-                    const int stage = kcnt % p.stages, ph = (kcnt / p.stages) & 1;
-                    const int g = (t - t0) & 1;  // softmax group that takes this key tile
-                    if (!mbar_wait(&full[stage], ph, abort_flag)) { ok = false; break; }
-                    for (int qb = 0; qb < nqt; ++qb, ++acnt[g]) {
+                int ti[kGroups] = {0, 1};   // next key tile (index within the split) of each group
+                int qb[kGroups] = {0, 0};   // next query tile of that key tile
+                uint32_t idle = 0;
+                while ((ti[0] < n_t || ti[1] < n_t) && ok) {
+                    bool progressed = false;
+#pragma unroll
+                    for (int g = 0; g < kGroups; ++g) {
+                        if (ti[g] >= n_t) continue;
+                        const int n = c * n_t + ti[g];  // position of the key tile in the load sequence
+                        const int stage = n % p.stages, ph = (n / p.stages) & 1;
                         const int buf = 2 * g + (acnt[g] & 1), bph = (acnt[g] >> 1) & 1;
-                        if (!mbar_wait(&acc_empty[buf], bph ^ 1, abort_flag)) { ok = false; break; }
+                        if (!mbar_test_wait(&full[stage], ph) || !mbar_test_wait(&acc_empty[buf], bph ^ 1)) continue;
                         tc_fence_after();
-                        const uint32_t qa = q_addr + qb * kTileBytes, ka = ring_addr + stage * kTileBytes;
+                        const uint32_t qa = q_addr + qb[g] * kTileBytes, ka = ring_addr + stage * kTileBytes;
                         const uint32_t a_addr = MODE == kLse ? qa : ka, b_addr = MODE == kLse ? ka : qa;
 #pragma unroll
                         for (int k = 0; k < D / 16; ++k) {
@@ -324,8 +333,23 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                                       smem_desc_sw128(b_addr + off), idesc, k > 0);
                         }
                         umma_commit(&acc_full[buf]);  // the accumulator is ready for its softmax group
+                        ++acnt[g];
+                        if (++qb[g] == nqt) {
+                            umma_commit(&empty[stage]);  // the stage may be refilled once these MMAs have read it
+                            qb[g] = 0;
+                            ti[g] += kGroups;
+                        }
+                        progressed = true;
                     }
-                    if (ok) umma_commit(&empty[stage]);  // the stage may be refilled once these MMAs have read it
+                    if (progressed) {
+                        idle = 0;
+                    } else if (++idle > 64) {
+                        if (*abort_flag || idle > kSpinLimit) {
+                            *abort_flag = 1;
+                            ok = false;
+                        }
+                        __nanosleep(32);
+                    }
                 }
                 if (ok) umma_commit(q_empty);
             }
