@@ -13,7 +13,10 @@ from typing import Optional, Sequence
 
 import numpy as np
 
-_LIB_PATH = Path(__file__).resolve().parent / "libfinch.so"
+import os
+
+# FINCH_LIB lets a developer load an alternative build of the library (same ABI) for experiments
+_LIB_PATH = Path(os.environ.get("FINCH_LIB") or Path(__file__).resolve().parent / "libfinch.so")
 _lib = None
 
 FINCH_OK = 0

@@ -301,7 +301,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         // =================================================================== MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_bf16_f32(kRows, kRows);
-            const uint32_t q_addr = smem_u32(q_res), ring_addr = smem_u32(k_ring);
+            const uint64_t q_desc = smem_desc_sw128(smem_u32(q_res)), ring_desc = smem_desc_sw128(smem_u32(k_ring));
             // The two softmax groups consume independent streams of accumulators (group g: key tiles t0 + g,
             // t0 + g + 2, .. of the split, every resident query tile of each).  The issuer serves whichever group
             // has a free accumulator and a loaded key tile, so neither group waits for the other's backlog.
@@ -324,13 +324,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                         const int buf = 2 * g + (acnt[g] & 1), bph = (acnt[g] >> 1) & 1;
                         if (!mbar_test_wait(&full[stage], ph) || !mbar_test_wait(&acc_empty[buf], bph ^ 1)) continue;
                         tc_fence_after();
-                        const uint32_t qa = q_addr + qb[g] * kTileBytes, ka = ring_addr + stage * kTileBytes;
-                        const uint32_t a_addr = MODE == kLse ? qa : ka, b_addr = MODE == kLse ? ka : qa;
+                        // one descriptor per operand tile; the K = 16 steps only advance its address field (a
+                        // lone thread issues these, so every instruction saved here is MMA issue rate gained)
+                        const uint64_t qd = q_desc + (uint64_t)((qb[g] * kTileBytes) >> 4);
+                        const uint64_t kd = ring_desc + (uint64_t)((stage * kTileBytes) >> 4);
+                        const uint64_t a_desc = MODE == kLse ? qd : kd, b_desc = MODE == kLse ? kd : qd;
+                        const uint32_t d_addr = tmem_base + buf * kRows;
 #pragma unroll
                         for (int k = 0; k < D / 16; ++k) {
-                            const uint32_t off = (k / 4) * kSlabBytes + (k % 4) * 32;
-                            umma_bf16(tmem_base + buf * kRows, smem_desc_sw128(a_addr + off),
-                                      smem_desc_sw128(b_addr + off), idesc, k > 0);
+                            const uint64_t off = (uint64_t)(((k / 4) * kSlabBytes + (k % 4) * 32) >> 4);
+                            if (k == 0)
+                                umma_bf16_first(d_addr, a_desc + off, b_desc + off, idesc);
+                            else
+                                umma_bf16_acc(d_addr, a_desc + off, b_desc + off, idesc);
                         }
                         umma_commit(&acc_full[buf]);  // the accumulator is ready for its softmax group
                         ++acnt[g];
@@ -343,12 +349,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                     }
                     if (progressed) {
                         idle = 0;
-                    } else if (++idle > 64) {
+                    } else if ((++idle & 1023u) == 0) {  // keep polling; look at the abort flag now and then
                         if (*abort_flag || idle > kSpinLimit) {
                             *abort_flag = 1;
                             ok = false;
                         }
-                        __nanosleep(32);
+                        if (idle > (1u << 16)) __nanosleep(64);
                     }
                 }
                 if (ok) umma_commit(q_empty);
@@ -453,7 +459,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         }
     }
 
-    // ---- common epilogue: everyone meets here, also after a timed-out wait
+    // ---- common epilogue: everyone meets here, also after a timed-out wait.  The role warps ran one lane only:
+    // bring each warp back together first, the CTA barrier must be executed by whole warps.
+    __syncwarp();
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, FINCH_DEV_TIMEOUT);

@@ -48,15 +48,17 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait: gives up after about a second (or as soon as another thread of the CTA has given up), raises
-// *abort_flag and returns false.  Callers then leave their loops and fall through to the common epilogue.
-constexpr uint32_t kSpinLimit = 1u << 22;
+// Bounded wait: polls (try_wait suspends the thread in hardware for a short while by itself) and gives up after
+// roughly a second, or as soon as another thread of the CTA has given up; it then raises *abort_flag and returns
+// false, and callers leave their loops for the common epilogue.  No software sleep on the fast path: a sleeping
+// waiter wakes too late for handshakes that complete in well under a microsecond.
+constexpr uint32_t kSpinLimit = 1u << 24;
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (it > 64) {
+        if ((it & 1023u) == 1023u) {
             if (*abort_flag) return false;
-            __nanosleep(it > 4096 ? 256 : 32);
+            if (it > (1u << 16)) __nanosleep(64);
         }
     }
     *abort_flag = 1;
@@ -98,6 +100,23 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The same without the run-time accumulate flag: the first K step overwrites D, the others add to it.
+__device__ __forceinline__ void umma_bf16_first(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc)
+        : "memory");
+}
+__device__ __forceinline__ void umma_bf16_acc(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.eq.b32 p, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc)
         : "memory");
 }
 // Arrive on an mbarrier once every tcgen05.mma issued so far by this thread has completed.
