@@ -100,6 +100,26 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
+// Packed pairs of fp32 (sm_100 executes these as one instruction on the FMA pipe).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
 // kLse: fold 32 columns (keys) of one accumulator row into the row's running (reference, sum of exp2).
 // The reference is the maximum of the row's first chunk, not the running maximum: any reference works as long as
 // the sum stays finite, and skipping the per-element maximum saves a quarter of the instructions.  If the sum
@@ -121,13 +141,20 @@ __device__ __forceinline__ void lse_chunk(const uint32_t (&r)[32], int nv, float
     }
     for (int attempt = 0; attempt < 8; ++attempt) {
         const float negm = -(m_raw * scale2);
-        float a0 = 0.f, a1 = 0.f;
+        const uint64_t s2 = pack2(scale2, scale2), n2 = pack2(negm, negm);
+        uint64_t acc0 = 0, acc1 = 0;  // two pairs of partial sums (+0.0f bit patterns)
 #pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-            a0 += ex2(fmaf(v[e], scale2, negm));
-            a1 += ex2(fmaf(v[e + 1], scale2, negm));
+        for (int e = 0; e < 32; e += 4) {
+            float x0, x1, x2, x3;
+            unpack2(fma2(pack2(v[e], v[e + 1]), s2, n2), x0, x1);
+            unpack2(fma2(pack2(v[e + 2], v[e + 3]), s2, n2), x2, x3);
+            acc0 = add2(acc0, pack2(ex2(x0), ex2(x1)));
+            acc1 = add2(acc1, pack2(ex2(x2), ex2(x3)));
         }
-        const float zn = z + (a0 + a1);
+        float a0, a1, a2, a3;
+        unpack2(acc0, a0, a1);
+        unpack2(acc1, a2, a3);
+        const float zn = z + ((a0 + a1) + (a2 + a3));
         if (!(zn > 3.0e38f)) {  // finite -- or NaN, on a lane that holds no prompt row: nothing to repair
             z = zn;
             break;
@@ -157,7 +184,8 @@ __device__ __forceinline__ void lse_accumulate(uint32_t taddr, int valid, float 
 }
 
 // kColsum: add to (c0, c1) the weights exp2(s * scale2 - ref_r) * w_r of one accumulator row (a key) over the valid
-// prompt rows of the query tile: v0 rows in its first 64-row half, v1 in its second.  sm[r] = (-ref_r, w_r).
+// prompt rows of the query tile: v0 rows in its first 64-row half, v1 in its second.  The statistics are staged
+// in pairs of rows, (-ref_a, -ref_b, w_a, w_b), so that one 128-bit load feeds two packed operations.
 __device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[32], int nv, float scale2, const float4 *sm4, float &c0,
                                              float &c1) {
     float v[32];
@@ -167,12 +195,16 @@ __device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[32], int nv, fl
 #pragma unroll
         for (int e = 0; e < 32; ++e) v[e] = e < nv ? v[e] : -INFINITY;  // rows past the prompt weigh nothing
     }
+    const uint64_t s2 = pack2(scale2, scale2);
+    uint64_t acc = pack2(c0, c1);
 #pragma unroll
     for (int e = 0; e < 32; e += 2) {
-        const float4 s4 = sm4[e / 2];  // statistics of two prompt rows
-        c0 = fmaf(ex2(fmaf(v[e], scale2, s4.x)), s4.y, c0);
-        c1 = fmaf(ex2(fmaf(v[e + 1], scale2, s4.z)), s4.w, c1);
+        const float4 s4 = sm4[e / 2];  // two prompt rows: (-ref_a, -ref_b, w_a, w_b)
+        float x0, x1;
+        unpack2(fma2(pack2(v[e], v[e + 1]), s2, pack2(s4.x, s4.y)), x0, x1);
+        acc = fma2(pack2(ex2(x0), ex2(x1)), pack2(s4.z, s4.w), acc);
     }
+    unpack2(acc, c0, c1);
 }
 
 __device__ __forceinline__ void colsum_accumulate(uint32_t taddr, int v0, int v1, float scale2, const float2 *sm,
@@ -430,7 +462,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                     float2 out = make_float2(0.f, 0.f);
                     if (r % kSub < sb.valid)
                         out = p.merged[((int64_t)u.l * mv.Hq + u.G * mv.hpg + sb.hh) * bv.total_q + u.q0 + sb.p0 + r % kSub];
-                    sm[idx] = out;
+                    // rows 2k and 2k+1 share one float4: (-ref_2k, -ref_2k+1, w_2k, w_2k+1)
+                    float *smf = (float *)sm + (idx >> 1) * 4 + (idx & 1);
+                    smf[0] = out.x;
+                    smf[2] = out.y;
                 }
                 __syncwarp();
                 for (int t = t0 + g; t < t1 && ok; t += kGroups) {
