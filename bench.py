@@ -175,12 +175,11 @@ def run_ours(args, cfg: wl.Config):
                       dev["chunk_pos"], batch, out_k, out_v, out_pos, kept, out_len, scores, ws)
 
     def step_e2e():
-        for k in ("q", "chunk_k", "chunk_v", "chunk_pos"):      # this step's inputs; the cache is carried on device
-            dev[k].copy_(host[k], non_blocking=True)
-        step()
-        kept_host.copy_(kept, non_blocking=True)                # the step's result: kept positions and lengths
-        len_host.copy_(out_len, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+        # this step's inputs come from pinned host memory through the C ABI's host-buffer call; the cache is
+        # carried on the device; the kept positions and lengths come back to the host
+        fb.finch_step_host(ctx, host["q"], host["chunk_k"], host["chunk_v"], host["chunk_pos"], dev["q"],
+                           dev["chunk_k"], dev["chunk_v"], dev["chunk_pos"], dev["cache_k"], dev["cache_v"],
+                           dev["cache_pos"], batch, out_k, out_v, out_pos, kept, out_len, kept_host, len_host, ws)
 
     def timed(fn, n):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

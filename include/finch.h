@@ -17,7 +17,7 @@
  *    only the context and one 4-byte device status word and frees only those.
  *  - Work is enqueued asynchronously on `cuda_stream` (a cudaStream_t passed as
  *    void*; NULL = the legacy default stream).  No call synchronises except
- *    finch_device_status.
+ *    finch_device_status and finch_step_host.
  *  - Arguments are validated on the host; a call that returns anything but FINCH_OK
  *    has enqueued nothing.  Nothing throws or aborts across this boundary.  Kernels
  *    never trap: device-side anomalies (inconsistent batch metadata, a bounded wait
@@ -186,6 +186,24 @@ finch_status finch_step(finch_ctx *ctx, const finch_tensor *prompt_q, const finc
                         const finch_tensor *chunk_v, const int32_t *chunk_pos, const finch_batch *batch,
                         const finch_tensor *out_k, const finch_tensor *out_v, int32_t *out_pos, int32_t *kept_idx,
                         int32_t *out_len, float *scores, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* The same step for a caller whose new inputs live in HOST memory (the end-to-end path: the paper's chunk loop,
+ * Section "Method", "Document Segmentation", feeds one chunk per step).  host_prompt_q, host_chunk_k, host_chunk_v
+ * are dense [n_layers][heads][tokens][head_dim] arrays and host_chunk_pos a dense [total_chunk] array, preferably in
+ * pinned memory; they are copied into the caller's DEVICE staging tensors stage_* (which must be dense and of the
+ * same shapes), the step runs on them and on the device-resident cache, and kept_idx / out_len are copied back to
+ * host_kept_idx [n_layers][G][total_cache] / host_out_len [batch].  The compressed cache (out_k, out_v, out_pos)
+ * stays on the device for the next step.  Unlike the other calls this one WAITS for the stream before it returns.
+ * The workspace must hold finch_workspace_bytes (scores live there).  Errors as for finch_step, plus
+ * FINCH_ERR_BAD_LAYOUT when a staging tensor is not dense. */
+finch_status finch_step_host(finch_ctx *ctx, const void *host_prompt_q, const void *host_chunk_k,
+                             const void *host_chunk_v, const int32_t *host_chunk_pos, const finch_tensor *stage_q,
+                             const finch_tensor *stage_chunk_k, const finch_tensor *stage_chunk_v,
+                             int32_t *stage_chunk_pos, const finch_tensor *cache_k, const finch_tensor *cache_v,
+                             const int32_t *cache_pos, const finch_batch *batch, const finch_tensor *out_k,
+                             const finch_tensor *out_v, int32_t *out_pos, int32_t *kept_idx, int32_t *out_len,
+                             int32_t *host_kept_idx, int32_t *host_out_len, void *ws, size_t ws_bytes,
+                             void *cuda_stream);
 
 /* Synchronises `cuda_stream`, copies the status word to *out (host) and clears it.  Returns FINCH_ERR_DEVICE_STATUS
  * when the word was non-zero, FINCH_ERR_CUDA when the stream reports an error. */

@@ -32,7 +32,7 @@ FINCH_GROUP_PER_KV_HEAD, FINCH_GROUP_PER_LAYER = 0, 1
 FINCH_DEV_BAD_BATCH, FINCH_DEV_TIMEOUT, FINCH_DEV_BAD_INDEX = 1, 2, 4
 
 EXPORTS = ("finch_ctx_create", "finch_ctx_destroy", "finch_workspace_bytes", "finch_score", "finch_select",
-           "finch_compact", "finch_step", "finch_device_status", "finch_launch_count", "finch_status_string", "finch_score_static", "finch_score_static_max_rows")
+           "finch_compact", "finch_step", "finch_device_status", "finch_launch_count", "finch_status_string", "finch_score_static", "finch_score_static_max_rows", "finch_step_host")
 
 
 class finch_config(C.Structure):
@@ -230,3 +230,18 @@ def finch_score_static(ctx, prompt_q, cache_k, chunk_k, batch: Batch, scores, ro
 
 def finch_score_static_max_rows() -> int:
     return int(load().finch_score_static_max_rows())
+
+
+def finch_step_host(ctx, host_prompt_q, host_chunk_k, host_chunk_v, host_chunk_pos, stage_q, stage_chunk_k,
+                    stage_chunk_v, stage_chunk_pos, cache_k, cache_v, cache_pos, batch: Batch, out_k, out_v, out_pos,
+                    kept_idx, out_len, host_kept_idx, host_out_len, ws, stream=None) -> None:
+    """finch_step with this step's inputs in host memory (torch CPU tensors, ideally pinned) and the kept indices
+    and lengths returned to host tensors; the call returns after the stream has finished."""
+    ts = [_tensor(t) for t in (stage_q, stage_chunk_k, stage_chunk_v, cache_k, cache_v, out_k, out_v)]
+    _check(load().finch_step_host(
+        ctx, C.c_void_p(_ptr(host_prompt_q)), C.c_void_p(_ptr(host_chunk_k)), C.c_void_p(_ptr(host_chunk_v)),
+        C.c_void_p(_ptr(host_chunk_pos)), C.byref(ts[0]), C.byref(ts[1]), C.byref(ts[2]),
+        C.c_void_p(_ptr(stage_chunk_pos)), C.byref(ts[3]), C.byref(ts[4]), C.c_void_p(_ptr(cache_pos)),
+        C.byref(batch.c), C.byref(ts[5]), C.byref(ts[6]), C.c_void_p(_ptr(out_pos)), C.c_void_p(_ptr(kept_idx)),
+        C.c_void_p(_ptr(out_len)), C.c_void_p(_ptr(host_kept_idx)), C.c_void_p(_ptr(host_out_len)),
+        C.c_void_p(_ptr(ws)), C.c_size_t(_nbytes(ws)), C.c_void_p(_stream(stream))), "finch_step_host")

@@ -285,6 +285,64 @@ finch_status finch_step(finch_ctx *ctx, const finch_tensor *prompt_q, const finc
     return cuda_status(e);
 }
 
+// finch_step with this step's new inputs in HOST memory: copies prompt_q, chunk_k, chunk_v and chunk_pos into the
+// caller's device staging tensors, runs the step, copies kept_idx and out_len back and waits for the stream.
+finch_status finch_step_host(finch_ctx *ctx, const void *host_prompt_q, const void *host_chunk_k,
+                             const void *host_chunk_v, const int32_t *host_chunk_pos, const finch_tensor *stage_q,
+                             const finch_tensor *stage_chunk_k, const finch_tensor *stage_chunk_v,
+                             int32_t *stage_chunk_pos, const finch_tensor *cache_k, const finch_tensor *cache_v,
+                             const int32_t *cache_pos, const finch_batch *batch, const finch_tensor *out_k,
+                             const finch_tensor *out_v, int32_t *out_pos, int32_t *kept_idx, int32_t *out_len,
+                             int32_t *host_kept_idx, int32_t *host_out_len, void *ws, size_t ws_bytes,
+                             void *cuda_stream) {
+    finch_status s = check_batch(ctx, batch);
+    if (s) return s;
+    if (!stage_q || !stage_chunk_k || !stage_chunk_v) return FINCH_ERR_INVALID_ARG;
+    const ModelView &mv = ctx->model;
+    auto dense = [&](const finch_tensor *t, int heads, int64_t tokens) {
+        return t->stride_tok == mv.d && t->stride_head == tokens * mv.d && t->stride_layer == (int64_t)heads * tokens * mv.d;
+    };
+    if (!dense(stage_q, mv.Hq, batch->total_q) || !dense(stage_chunk_k, mv.Hkv, batch->total_chunk) ||
+        !dense(stage_chunk_v, mv.Hkv, batch->total_chunk))
+        return FINCH_ERR_BAD_LAYOUT;  // the staging tensors receive dense host arrays
+    if (batch->total_q > 0 && !host_prompt_q) return FINCH_ERR_INVALID_ARG;
+    if (batch->total_chunk > 0 && (!host_chunk_k || !host_chunk_v || !host_chunk_pos || !stage_chunk_pos))
+        return FINCH_ERR_INVALID_ARG;
+    if (batch->batch > 0 && !host_out_len) return FINCH_ERR_INVALID_ARG;
+    if (batch->total_cache > 0 && !host_kept_idx) return FINCH_ERR_INVALID_ARG;
+    // validate the step itself before anything is enqueued (a validation-only context stops here)
+    if ((s = validate_score(ctx, stage_q, cache_k, stage_chunk_k, batch))) return s;
+    if ((s = validate_compact(ctx, kept_idx, out_len, cache_k, cache_v, cache_pos, stage_chunk_k, stage_chunk_v,
+                              stage_chunk_pos, batch, out_k, out_v, out_pos)))
+        return s;
+    if (!ws) return FINCH_ERR_INVALID_ARG;
+    if (ws_bytes < ws_layout(ctx, batch).total) return FINCH_ERR_WORKSPACE_TOO_SMALL;
+    if (ctx->dry) return FINCH_ERR_UNSUPPORTED;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const size_t e = mv.elem_bytes;
+    const size_t q_bytes = (size_t)mv.L * mv.Hq * batch->total_q * mv.d * e;
+    const size_t c_bytes = (size_t)mv.L * mv.Hkv * batch->total_chunk * mv.d * e;
+    cudaError_t ce = cudaSuccess;
+    if (q_bytes) ce = cudaMemcpyAsync(stage_q->ptr, host_prompt_q, q_bytes, cudaMemcpyHostToDevice, stream);
+    if (ce == cudaSuccess && c_bytes)
+        ce = cudaMemcpyAsync(stage_chunk_k->ptr, host_chunk_k, c_bytes, cudaMemcpyHostToDevice, stream);
+    if (ce == cudaSuccess && c_bytes)
+        ce = cudaMemcpyAsync(stage_chunk_v->ptr, host_chunk_v, c_bytes, cudaMemcpyHostToDevice, stream);
+    if (ce == cudaSuccess && batch->total_chunk)
+        ce = cudaMemcpyAsync(stage_chunk_pos, host_chunk_pos, (size_t)batch->total_chunk * 4, cudaMemcpyHostToDevice,
+                             stream);
+    if (ce != cudaSuccess) return FINCH_ERR_CUDA;
+    s = finch_step(ctx, stage_q, cache_k, cache_v, cache_pos, stage_chunk_k, stage_chunk_v, stage_chunk_pos, batch, out_k,
+                   out_v, out_pos, kept_idx, out_len, nullptr, ws, ws_bytes, cuda_stream);
+    if (s) return s;
+    const size_t kept_bytes = (size_t)mv.L * mv.G * batch->total_cache * 4;
+    if (kept_bytes) ce = cudaMemcpyAsync(host_kept_idx, kept_idx, kept_bytes, cudaMemcpyDeviceToHost, stream);
+    if (ce == cudaSuccess && batch->batch)
+        ce = cudaMemcpyAsync(host_out_len, out_len, (size_t)batch->batch * 4, cudaMemcpyDeviceToHost, stream);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
+    return cuda_status(ce);
+}
+
 finch_status finch_launch_count(const finch_ctx *ctx, uint64_t *out) {
     if (!ctx || !out) return FINCH_ERR_INVALID_ARG;
     *out = ctx->launches;

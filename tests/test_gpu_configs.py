@@ -253,3 +253,43 @@ def test_chunk_loop_on_gpu_matches_oracle_and_keeps_planted_keys():
         for l in range(L):
             for g in range(cfg.n_groups):
                 assert planted[b] <= set(final[l, g, cache_off[b]:cache_off[b] + cache_len[b]].tolist())
+
+
+def test_step_host_matches_step():
+    """finch_step_host (inputs in pinned host memory, results read back) against finch_step on resident inputs."""
+    import torch
+    cfg = wl.scaled(wl.CONFIGS["c3"], n_layers=2, n_q_heads=8, n_kv_heads=2, head_dim=128,
+                    requests=(wl.Request(128, 9999, 300, 200), wl.Request(40, 9999, 70, 90)))
+    st = wl.steady_state(cfg, [0, 1], step=2)
+    g = GpuStep(cfg, st, 2)
+    try:
+        g.run(scores=False)
+        assert g.status() == 0
+        want = g.results()
+        host = {k: to_device(st[k], "bf16", "cpu").pin_memory() for k in ("q", "chunk_k", "chunk_v")}
+        host_pos = torch.from_numpy(st["chunk_pos"]).pin_memory()
+        stage = {k: torch.zeros_like(getattr(g, k)) for k in ("q", "chunk_k", "chunk_v")}
+        stage_pos = torch.zeros_like(g.chunk_pos)
+        out_k, out_v = torch.zeros_like(g.out_k), torch.zeros_like(g.out_v)
+        out_pos, kept, out_len = torch.full_like(g.out_pos, -1), torch.full_like(g.kept_idx, -1), torch.zeros_like(g.out_len)
+        host_kept = torch.full(kept.shape, -5, dtype=torch.int32).pin_memory()
+        host_len = torch.full(out_len.shape, -5, dtype=torch.int32).pin_memory()
+        for _ in range(2):
+            fb.finch_step_host(g.ctx, host["q"], host["chunk_k"], host["chunk_v"], host_pos, stage["q"],
+                               stage["chunk_k"], stage["chunk_v"], stage_pos, g.cache_k, g.cache_v, g.cache_pos,
+                               g.batch, out_k, out_v, out_pos, kept, out_len, host_kept, host_len, g.ws)
+            assert g.status() == 0
+            np.testing.assert_array_equal(host_len.numpy(), want["out_len"])
+            np.testing.assert_array_equal(host_kept.numpy(), want["kept_idx"])
+            np.testing.assert_array_equal(to_host(out_k, "bf16"), want["out_k"])
+            np.testing.assert_array_equal(to_host(out_v, "bf16"), want["out_v"])
+            np.testing.assert_array_equal(out_pos.cpu().numpy(), want["out_pos"])
+        # a staging tensor that is not dense is refused before anything is copied
+        padded = torch.zeros((2, 8, g.q.shape[2], 256), dtype=torch.bfloat16, device="cuda")[:, :, :, :128]
+        with pytest.raises(fb.FinchError) as e:
+            fb.finch_step_host(g.ctx, host["q"], host["chunk_k"], host["chunk_v"], host_pos, padded,
+                               stage["chunk_k"], stage["chunk_v"], stage_pos, g.cache_k, g.cache_v, g.cache_pos,
+                               g.batch, out_k, out_v, out_pos, kept, out_len, host_kept, host_len, g.ws)
+        assert e.value.status == fb.FINCH_ERR_BAD_LAYOUT
+    finally:
+        g.close()
