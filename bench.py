@@ -51,9 +51,10 @@ def step_counts(cfg: wl.Config, st: dict) -> dict:
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons sampled while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """nvidia-smi clocks and throttle reasons, sampled in the background and filtered to a wall-clock window."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_index: int):
         self.proc, self.gpu = None, gpu_index
@@ -66,7 +67,9 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
-    def stop(self) -> dict:
+    def stop(self, t_begin: float, t_end: float) -> dict:
+        """Summary of the samples taken between the two time.time() stamps (all samples if none fall inside)."""
+        import datetime
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -75,17 +78,23 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.proc.kill()
             out, _ = self.proc.communicate()
-        sm, mx, reasons = [], None, set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        rows = []
         for line in out.splitlines():
             f = [x.strip() for x in line.split(",")]
-            if len(f) < 6 or not f[0].isdigit():
+            if len(f) < 7 or not f[1].isdigit():
                 continue
-            sm.append(int(f[0]))
-            mx = int(f[1])
-            reasons |= {n for n, v in zip(names, f[2:6]) if v == "Active"}
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
-                "samples": len(sm)}
+            try:
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+            except ValueError:
+                ts = None
+            rows.append((ts, int(f[1]), int(f[2]), {n for n, v in zip(names, f[3:7]) if v == "Active"}))
+        inside = [r for r in rows if r[0] is not None and t_begin <= r[0] <= t_end]
+        use = inside or rows
+        reasons = set().union(*[r[3] for r in use]) if use else set()
+        return {"sm_mhz": statistics.median([r[1] for r in use]) if use else None,
+                "sm_max_mhz": use[0][2] if use else None, "reasons": sorted(reasons), "samples": len(use),
+                "window": "timed steps" if inside else "whole run (no sample fell inside the timed steps)"}
 
 
 def dist_env():
@@ -142,6 +151,8 @@ def run_ours(args, cfg: wl.Config):
     fbuild.build()
     fb.load()
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()               # started early: nvidia-smi needs a moment before its first sample
     layers = list(range(cfg.n_layers))
     st = wl.steady_state(cfg, layers)
     counts = step_counts(cfg, st)
@@ -195,13 +206,13 @@ def run_ours(args, cfg: wl.Config):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / n
 
-    sampler = ClockSampler(local_rank)
-    sampler.start()               # runs through warm-up, the timed steps and the per-phase loop: all under load
     for _ in range(max(args.warmup, 3)):
         step()
     assert fb.finch_device_status(ctx) == 0
     launches0 = fb.finch_launch_count(ctx)
+    t_begin = time.time()
     ms_local = timed(step, args.steps)
+    t_end = time.time()
     launches = fb.finch_launch_count(ctx) - launches0
     assert fb.finch_device_status(ctx) == 0
     ms, tokens = aggregate_over_ranks(ms_local, counts["tokens"], world, "nccl")
@@ -221,7 +232,7 @@ def run_ours(args, cfg: wl.Config):
         torch.cuda.synchronize()
         phase += [ev[i].elapsed_time(ev[i + 1]) for i in range(3)]
     phase /= args.steps
-    clocks = sampler.stop()
+    clocks = sampler.stop(t_begin, t_end)
 
     step_e2e()
     ms_e2e_local = timed(step_e2e, max(1, min(args.steps, 5)))
@@ -281,7 +292,7 @@ def run_reference(args, cfg: wl.Config):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="c3", choices=sorted(wl.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

@@ -42,21 +42,37 @@ compact_kernel(ModelView mv, BatchView bv, const int *kept_idx, const int *out_l
 
     const int pieces = mv.d * mv.elem_bytes / 16;  // 16-byte pieces per row
     const int per_row = pieces * 2 * mv.kvpg;      // K and V, every KV head of the group
-    for (int e = threadIdx.x; e < rows * per_row; e += kCompactThreads) {
-        const int row = e / per_row, rem = e % per_row;
-        const int piece = rem % pieces, which = rem / pieces;  // which = kv * 2 + {0: K, 1: V}
+    // A warp owns 32 consecutive pieces of an output row (fully coalesced) and walks the CTA's rows eight apart;
+    // everything that does not depend on the row is computed once per thread, outside the row loop.
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    constexpr int kRowsInFlight = kCompactThreads / 32;
+    for (int cs = tx; cs < per_row; cs += 32) {
+        const int piece = cs % pieces, which = cs / pieces;  // which = kv * 2 + {0: K, 1: V}
         const int kvh = u.G * mv.kvpg + which / 2;
         const bool is_v = which & 1;
-        const int j = src_idx[row];
-        if (j < 0) continue;
-        const TensorView &src = j < u.c ? (is_v ? cache_v : cache_k) : (is_v ? chunk_v : chunk_k);
-        const int64_t src_tok = j < u.c ? u.cache0 + j : u.chunk0 + j - u.c;
+        const TensorView &ca = is_v ? cache_v : cache_k;
+        const TensorView &ch = is_v ? chunk_v : chunk_k;
         const TensorView &dst = is_v ? out_v : out_k;
-        const int64_t se = (int64_t)u.l * src.stride_layer + (int64_t)kvh * src.stride_head + src_tok * src.stride_tok;
-        const int64_t de = (int64_t)u.l * dst.stride_layer + (int64_t)kvh * dst.stride_head +
-                           (int64_t)(u.cache0 + i0 + row) * dst.stride_tok;
-        const uint4 v = __ldg((const uint4 *)(src.ptr + se * mv.elem_bytes) + piece);
-        ((uint4 *)(const_cast<char *>(dst.ptr) + de * mv.elem_bytes))[piece] = v;
+        const int64_t e = mv.elem_bytes;
+        const char *ca_base = ca.ptr + ((int64_t)u.l * ca.stride_layer + (int64_t)kvh * ca.stride_head +
+                                        (int64_t)u.cache0 * ca.stride_tok) * e + piece * 16;
+        const char *ch_base = ch.ptr + ((int64_t)u.l * ch.stride_layer + (int64_t)kvh * ch.stride_head +
+                                        (int64_t)(u.chunk0 - u.c) * ch.stride_tok) * e + piece * 16;
+        char *dst_base = const_cast<char *>(dst.ptr) + ((int64_t)u.l * dst.stride_layer + (int64_t)kvh * dst.stride_head +
+                                                        (int64_t)(u.cache0 + i0) * dst.stride_tok) * e + piece * 16;
+        const int64_t ca_step = ca.stride_tok * e, ch_step = ch.stride_tok * e, dst_step = dst.stride_tok * e;
+        uint4 v[kRowsPerCta / kRowsInFlight];
+#pragma unroll
+        for (int k = 0; k < kRowsPerCta / kRowsInFlight; ++k) {  // all of this thread's loads first ..
+            const int row = ty + k * kRowsInFlight;
+            const int j = row < rows ? src_idx[row] : -1;
+            if (j >= 0) v[k] = __ldg((const uint4 *)(j < u.c ? ca_base + j * ca_step : ch_base + j * ch_step));
+        }
+#pragma unroll
+        for (int k = 0; k < kRowsPerCta / kRowsInFlight; ++k) {  // .. then its stores
+            const int row = ty + k * kRowsInFlight;
+            if (row < rows && src_idx[row] >= 0) *(uint4 *)(dst_base + row * dst_step) = v[k];
+        }
     }
 }
 
