@@ -52,6 +52,7 @@ struct TcParams {
     int splits;        // key splits per unit (grid x)
     int stages;        // key-tile ring depth that fits beside the resident queries
     int q_tiles;       // query tiles resident at a time (1..4), sized from the batch's longest prompt
+    int n_items;       // work items = splits x units x requests, walked by a persistent grid
 };
 
 struct KeyTile {
@@ -227,6 +228,41 @@ __device__ __forceinline__ void colsum_accumulate(uint32_t taddr, int v0, int v1
     }
 }
 
+// One work item = one key split of one unit.  A CTA walks a contiguous range of items (split fastest), so that
+// consecutive items usually belong to the same unit and the resident query tiles can stay where they are.
+struct Item {
+    UnitInfo u;
+    int key;  // identifies (unit, request): items with equal keys share their query tiles
+    int split, t0, t1, tps, k_tiles;
+    int sbq, n_sb, n_qt, n_chunks;
+    bool run;
+};
+
+__device__ __forceinline__ Item decode_item(const TcParams &p, int w, bool report) {
+    Item it;
+    const int units = p.mv.L * p.mv.G;
+    it.split = w % p.splits;
+    it.key = w / p.splits;
+    it.u = unit_info(p.mv, p.bv, it.key % units, it.key / units);
+    it.run = false;
+    if (!it.u.ok) {
+        if (report) atomicOr(p.status, FINCH_DEV_BAD_BATCH);
+        return it;
+    }
+    if (it.u.n_q < p.min_q || it.u.N == 0) return it;
+    it.k_tiles = n_key_tiles(it.u);
+    it.tps = (it.k_tiles + p.splits - 1) / p.splits;  // key tiles per split
+    it.t0 = it.split * it.tps;
+    it.t1 = min(it.k_tiles, it.t0 + it.tps);
+    if (it.t0 >= it.t1) return it;
+    it.sbq = (it.u.n_q + kSub - 1) / kSub;  // sub-blocks per query head
+    it.n_sb = p.mv.hpg * it.sbq;
+    it.n_qt = (it.n_sb + 1) / 2;  // query tiles of the group
+    it.n_chunks = (it.n_qt + p.q_tiles - 1) / p.q_tiles;
+    it.run = true;
+    return it;
+}
+
 template <int MODE, int D>
 __global__ void __launch_bounds__(kTcThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap cache_map,
@@ -240,39 +276,24 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     uint8_t *k_ring = smem + p.q_tiles * kTileBytes;
     uint8_t *aux = k_ring + p.stages * kTileBytes;
     uint64_t *q_full = (uint64_t *)aux;
-    uint64_t *q_empty = q_full + 1;
-    uint64_t *full = q_empty + 1;
+    uint64_t *full = q_full + 1;
     uint64_t *empty = full + kMaxStages;
     uint64_t *acc_full = empty + kMaxStages;
     uint64_t *acc_empty = acc_full + kAccBufs;
     uint32_t *tmem_slot = (uint32_t *)(acc_empty + kAccBufs);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
-    float2 *stats_sm = (float2 *)(aux + 1024);  // [4 softmax warps][q_tiles * 128] (-max, 1/sum), kColsum only
+    float2 *stats_sm = (float2 *)(aux + 1024);  // [8 softmax warps][q_tiles * 128] row statistics, kColsum only
 
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
-    const UnitInfo u = unit_info(mv, bv, blockIdx.y, blockIdx.z);
-    if (!u.ok) {
-        if (threadIdx.x == 0) atomicOr(p.status, FINCH_DEV_BAD_BATCH);
-        return;
-    }
-    if (u.n_q < p.min_q || u.N == 0) return;
-    const int kvh = u.G;  // one KV head per selection group on this path
-    const int k_tiles = n_key_tiles(u);
-    const int tps = (k_tiles + p.splits - 1) / p.splits;  // key tiles per split
-    const int split = blockIdx.x;
-    const int t0 = split * tps, t1 = min(k_tiles, t0 + tps);
-    if (t0 >= t1) return;
-    const int sbq = (u.n_q + kSub - 1) / kSub;  // sub-blocks per query head
-    const int n_sb = mv.hpg * sbq;
-    const int n_qt = (n_sb + 1) / 2;            // query tiles of the group
-    const int n_chunks = (n_qt + p.q_tiles - 1) / p.q_tiles;
+    // this CTA's contiguous range of work items
+    const int w0 = (int)((int64_t)blockIdx.x * p.n_items / gridDim.x);
+    const int w1 = (int)((int64_t)(blockIdx.x + 1) * p.n_items / gridDim.x);
     const int64_t rows_total = (int64_t)mv.L * mv.Hq * bv.total_q;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
-        mbar_init(q_empty, 1);
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
@@ -293,39 +314,61 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    // Every role walks the same items and keeps the same running counters (key tiles loaded, query loads,
+    // accumulators per group), so barrier phases stay in step across items without any extra handshake.
     if (warp == 0) {
         // =================================================================== TMA producer
         if (lane == 0) {
             prefetch_tensormap(&q_map);
             prefetch_tensormap(&cache_map);
             prefetch_tensormap(&chunk_map);
-            int kcnt = 0, q_issued = 0;
+            int kcnt = 0, qcnt = 0, pst = 0, pph = 0, last_stage = 0, last_ph = 0, prev_stage = 0, prev_ph = 0, q_key = -1;
             bool ok = true;
-            for (int c = 0; c < n_chunks && ok; ++c) {
-                const int qt0 = c * p.q_tiles;
-                const int nload = min(2 * min(p.q_tiles, n_qt - qt0), n_sb - 2 * qt0);
-                if (!mbar_wait(q_empty, (c & 1) ^ 1, abort_flag)) break;  // the previous chunk's MMAs have read it
-                mbar_expect_tx(q_full, nload * kSlabs * kSubBytes);
-                for (int sl = 0; sl < nload; ++sl) {
-                    const SubBlock sb = sub_block(2 * qt0 + sl, sbq, n_sb, u.n_q);
-                    uint8_t *dst = q_res + (sl / 2) * kTileBytes + (sl % 2) * kSubBytes;
-                    for (int s = 0; s < kSlabs; ++s)
-                        tma_load_4d(dst + s * kSlabBytes, &q_map, q_full, s * 64, u.q0 + sb.p0, u.G * mv.hpg + sb.hh, u.l);
-                }
-                ++q_issued;
-                for (int t = t0; t < t1; ++t, ++kcnt) {
-                    const int stage = kcnt % p.stages, ph = (kcnt / p.stages) & 1;
-                    if (!mbar_wait(&empty[stage], ph ^ 1, abort_flag)) { ok = false; break; }
-                    mbar_expect_tx(&full[stage], kTileBytes);
-                    const KeyTile kt = key_tile(u, t);
-                    const CUtensorMap *m = kt.is_chunk ? &chunk_map : &cache_map;
-                    for (int s = 0; s < kSlabs; ++s)
-                        tma_load_4d(k_ring + stage * kTileBytes + s * kSlabBytes, m, &full[stage], s * 64, kt.row0, kvh,
-                                    u.l);
+            for (int w = w0; w < w1 && ok; ++w) {
+                const Item it = decode_item(p, w, true);
+                if (!it.run) continue;
+                const UnitInfo &u = it.u;
+                for (int c = 0; c < it.n_chunks && ok; ++c) {
+                    if (!(it.n_chunks == 1 && q_key == it.key)) {  // the resident query tiles are not this item's
+                        // every MMA of the previous work must have read them.  The two groups' streams are issued
+                        // in no fixed order, so wait for the release of the last key tile of each (the last two loaded)
+                        if (kcnt > 1 && !mbar_wait(&empty[prev_stage], prev_ph, abort_flag)) { ok = false; break; }
+                        if (kcnt > 0 && !mbar_wait(&empty[last_stage], last_ph, abort_flag)) { ok = false; break; }
+                        const int qt0 = c * p.q_tiles;
+                        const int nload = min(2 * min(p.q_tiles, it.n_qt - qt0), it.n_sb - 2 * qt0);
+                        mbar_expect_tx(q_full, nload * kSlabs * kSubBytes);
+                        for (int sl = 0; sl < nload; ++sl) {
+                            const SubBlock sb = sub_block(2 * qt0 + sl, it.sbq, it.n_sb, u.n_q);
+                            uint8_t *dst = q_res + (sl / 2) * kTileBytes + (sl % 2) * kSubBytes;
+                            for (int s = 0; s < kSlabs; ++s)
+                                tma_load_4d(dst + s * kSlabBytes, &q_map, q_full, s * 64, u.q0 + sb.p0,
+                                            u.G * mv.hpg + sb.hh, u.l);
+                        }
+                        ++qcnt;
+                        q_key = it.n_chunks == 1 ? it.key : -1;
+                    }
+                    for (int t = it.t0; t < it.t1; ++t, ++kcnt) {
+                        const int stage = pst, ph = pph;
+                        if (++pst == p.stages) {
+                            pst = 0;
+                            pph ^= 1;
+                        }
+                        if (!mbar_wait(&empty[stage], ph ^ 1, abort_flag)) { ok = false; break; }
+                        mbar_expect_tx(&full[stage], kTileBytes);
+                        const KeyTile kt = key_tile(u, t);
+                        const CUtensorMap *m = kt.is_chunk ? &chunk_map : &cache_map;
+                        for (int s = 0; s < kSlabs; ++s)
+                            tma_load_4d(k_ring + stage * kTileBytes + s * kSlabBytes, m, &full[stage], s * 64, kt.row0,
+                                        u.G, u.l);
+                        prev_stage = last_stage;
+                        prev_ph = last_ph;
+                        last_stage = stage;
+                        last_ph = ph;
+                    }
                 }
             }
             // no copy may still be in flight when the CTA retires: wait (bounded) for the last loads issued
-            if (q_issued) mbar_wait(q_full, (q_issued - 1) & 1, abort_flag);
+            if (qcnt) mbar_wait(q_full, (qcnt - 1) & 1, abort_flag);
             for (int i = max(0, kcnt - p.stages); i < kcnt; ++i)
                 mbar_wait(&full[i % p.stages], (i / p.stages) & 1, abort_flag);
         }
@@ -337,59 +380,79 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             // The two softmax groups consume independent streams of accumulators (group g: key tiles t0 + g,
             // t0 + g + 2, .. of the split, every resident query tile of each).  The issuer serves whichever group
             // has a free accumulator and a loaded key tile, so neither group waits for the other's backlog.
-            const int n_t = t1 - t0;
             bool ok = true;
+            int kn = 0, qcnt = 0, q_key = -1;
             int acnt[kGroups] = {0, 0};
-            for (int c = 0; c < n_chunks && ok; ++c) {
-                const int nqt = min(p.q_tiles, n_qt - c * p.q_tiles);
-                if (!mbar_wait(q_full, c & 1, abort_flag)) break;
-                int ti[kGroups] = {0, 1};   // next key tile (index within the split) of each group
-                int qb[kGroups] = {0, 0};   // next query tile of that key tile
-                uint32_t idle = 0;
-                while ((ti[0] < n_t || ti[1] < n_t) && ok) {
-                    bool progressed = false;
+            for (int w = w0; w < w1 && ok; ++w) {
+                const Item it = decode_item(p, w, false);
+                if (!it.run) continue;
+                const int n_t = it.t1 - it.t0;
+                for (int c = 0; c < it.n_chunks && ok; ++c, kn += n_t) {
+                    const int nqt = min(p.q_tiles, it.n_qt - c * p.q_tiles);
+                    if (!(it.n_chunks == 1 && q_key == it.key)) {
+                        if (!mbar_wait(q_full, qcnt & 1, abort_flag)) { ok = false; break; }
+                        ++qcnt;
+                        q_key = it.n_chunks == 1 ? it.key : -1;
+                    }
+                    int ti[kGroups] = {0, 1};  // next key tile (index within the split) of each group
+                    int qb[kGroups] = {0, 0};  // next query tile of that key tile
+                    // ring stage and phase of each group's next key tile, kept incrementally: this lone thread
+                    // cannot afford an integer division per poll
+                    int st[kGroups], sph[kGroups];
 #pragma unroll
                     for (int g = 0; g < kGroups; ++g) {
-                        if (ti[g] >= n_t) continue;
-                        const int n = c * n_t + ti[g];  // position of the key tile in the load sequence
-                        const int stage = n % p.stages, ph = (n / p.stages) & 1;
-                        const int buf = 2 * g + (acnt[g] & 1), bph = (acnt[g] >> 1) & 1;
-                        if (!mbar_test_wait(&full[stage], ph) || !mbar_test_wait(&acc_empty[buf], bph ^ 1)) continue;
-                        tc_fence_after();
-                        // one descriptor per operand tile; the K = 16 steps only advance its address field (a
-                        // lone thread issues these, so every instruction saved here is MMA issue rate gained)
-                        const uint64_t qd = q_desc + (uint64_t)((qb[g] * kTileBytes) >> 4);
-                        const uint64_t kd = ring_desc + (uint64_t)((stage * kTileBytes) >> 4);
-                        const uint64_t a_desc = MODE == kLse ? qd : kd, b_desc = MODE == kLse ? kd : qd;
-                        const uint32_t d_addr = tmem_base + buf * kRows;
-#pragma unroll
-                        for (int k = 0; k < D / 16; ++k) {
-                            const uint64_t off = (uint64_t)(((k / 4) * kSlabBytes + (k % 4) * 32) >> 4);
-                            if (k == 0)
-                                umma_bf16_first(d_addr, a_desc + off, b_desc + off, idesc);
-                            else
-                                umma_bf16_acc(d_addr, a_desc + off, b_desc + off, idesc);
-                        }
-                        umma_commit(&acc_full[buf]);  // the accumulator is ready for its softmax group
-                        ++acnt[g];
-                        if (++qb[g] == nqt) {
-                            umma_commit(&empty[stage]);  // the stage may be refilled once these MMAs have read it
-                            qb[g] = 0;
-                            ti[g] += kGroups;
-                        }
-                        progressed = true;
+                        st[g] = (kn + g) % p.stages;
+                        sph[g] = ((kn + g) / p.stages) & 1;
                     }
-                    if (progressed) {
-                        idle = 0;
-                    } else if ((++idle & 1023u) == 0) {  // keep polling; look at the abort flag now and then
-                        if (*abort_flag || idle > kSpinLimit) {
-                            *abort_flag = 1;
-                            ok = false;
+                    uint32_t idle = 0;
+                    while ((ti[0] < n_t || ti[1] < n_t) && ok) {
+                        bool progressed = false;
+#pragma unroll
+                        for (int g = 0; g < kGroups; ++g) {
+                            if (ti[g] >= n_t) continue;
+                            const int stage = st[g];
+                            const int buf = 2 * g + (acnt[g] & 1), bph = (acnt[g] >> 1) & 1;
+                            if (!mbar_test_wait(&full[stage], sph[g]) || !mbar_test_wait(&acc_empty[buf], bph ^ 1))
+                                continue;
+                            tc_fence_after();
+                            // one descriptor per operand tile; the K = 16 steps only advance its address field
+                            const uint64_t qd = q_desc + (uint64_t)((qb[g] * kTileBytes) >> 4);
+                            const uint64_t kd = ring_desc + (uint64_t)((stage * kTileBytes) >> 4);
+                            const uint64_t a_desc = MODE == kLse ? qd : kd, b_desc = MODE == kLse ? kd : qd;
+                            const uint32_t d_addr = tmem_base + buf * kRows;
+#pragma unroll
+                            for (int k = 0; k < D / 16; ++k) {
+                                const uint64_t off = (uint64_t)(((k / 4) * kSlabBytes + (k % 4) * 32) >> 4);
+                                if (k == 0)
+                                    umma_bf16_first(d_addr, a_desc + off, b_desc + off, idesc);
+                                else
+                                    umma_bf16_acc(d_addr, a_desc + off, b_desc + off, idesc);
+                            }
+                            umma_commit(&acc_full[buf]);  // the accumulator is ready for its softmax group
+                            ++acnt[g];
+                            if (++qb[g] == nqt) {
+                                umma_commit(&empty[stage]);  // the stage may be refilled once these MMAs have read it
+                                qb[g] = 0;
+                                ti[g] += kGroups;
+                                st[g] += kGroups;
+                                while (st[g] >= p.stages) {
+                                    st[g] -= p.stages;
+                                    sph[g] ^= 1;
+                                }
+                            }
+                            progressed = true;
                         }
-                        if (idle > (1u << 16)) __nanosleep(64);
+                        if (progressed) {
+                            idle = 0;
+                        } else if ((++idle & 1023u) == 0) {  // keep polling; look at the abort flag now and then
+                            if (*abort_flag || idle > kSpinLimit) {
+                                *abort_flag = 1;
+                                ok = false;
+                            }
+                            if (idle > (1u << 16)) __nanosleep(64);
+                        }
                     }
                 }
-                if (ok) umma_commit(q_empty);
             }
         }
     } else {
@@ -399,95 +462,110 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         const int my_row = quarter * 32 + lane;  // row of the A tile this thread owns
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
         const float scale2 = mv.scale * kLog2e;
-        int acnt = 0;
+        int acnt = 0, q_key = -1;
         bool ok = true;
-        for (int c = 0; c < n_chunks && ok; ++c) {
-            const int qt0 = c * p.q_tiles;
-            const int nqt = min(p.q_tiles, n_qt - qt0);
-            if (MODE == kLse) {
-                float m_raw[kQTiles], z[kQTiles];
-                uint32_t live_mask = 0;  // bit qb: this thread's row of query tile qb holds a prompt row
+        for (int w = w0; w < w1 && ok; ++w) {
+            const Item it = decode_item(p, w, false);
+            if (!it.run) continue;
+            const UnitInfo &u = it.u;
+            const int t0 = it.t0, t1 = it.t1, sbq = it.sbq, n_sb = it.n_sb;
+            for (int c = 0; c < it.n_chunks && ok; ++c) {
+                const int qt0 = c * p.q_tiles;
+                const int nqt = min(p.q_tiles, it.n_qt - qt0);
+                const bool new_rows = !(it.n_chunks == 1 && q_key == it.key);
+                q_key = it.n_chunks == 1 ? it.key : -1;
+                if (MODE == kLse) {
+                    float m_raw[kQTiles], z[kQTiles];
+                    uint32_t live_mask = 0;  // bit qb: this thread's row of query tile qb holds a prompt row
 #pragma unroll
-                for (int k = 0; k < kQTiles; ++k) {
-                    m_raw[k] = -INFINITY;
-                    z[k] = 0.f;
-                    if (k < nqt && my_row % kSub < sub_block(2 * (qt0 + k) + my_row / kSub, sbq, n_sb, u.n_q).valid)
-                        live_mask |= 1u << k;
-                }
-                for (int t = t0 + g; t < t1 && ok; t += kGroups) {
-                    const KeyTile kt = key_tile(u, t);
-#pragma unroll 1
-                    for (int qb = 0; qb < nqt && ok; ++qb, ++acnt) {
-                        const int buf = 2 * g + (acnt & 1), bph = (acnt >> 1) & 1;
-                        // a wait's verdict is made warp-uniform so that a timeout takes the whole warp out
-                        if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[buf], bph, abort_flag))) { ok = false; break; }
-                        tc_fence_after();
-                        float mc = 0.f, zc = 0.f;  // the running statistics of query tile qb (kept in registers)
-#pragma unroll
-                        for (int k = 0; k < kQTiles; ++k)
-                            if (k == qb) {
-                                mc = m_raw[k];
-                                zc = z[k];
-                            }
-                        lse_accumulate(t_lane + buf * kRows, kt.valid, scale2, (live_mask >> qb) & 1u, mc, zc);
-#pragma unroll
-                        for (int k = 0; k < kQTiles; ++k)
-                            if (k == qb) {
-                                m_raw[k] = mc;
-                                z[k] = zc;
-                            }
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                    for (int k = 0; k < kQTiles; ++k) {
+                        m_raw[k] = -INFINITY;
+                        z[k] = 0.f;
+                        if (k < nqt && my_row % kSub < sub_block(2 * (qt0 + k) + my_row / kSub, sbq, n_sb, u.n_q).valid)
+                            live_mask |= 1u << k;
                     }
-                }
-                if (ok && t0 + g < t1) {
+                    for (int t = t0 + g; t < t1 && ok; t += kGroups) {
+                        const KeyTile kt = key_tile(u, t);
+#pragma unroll 1
+                        for (int qb = 0; qb < nqt && ok; ++qb, ++acnt) {
+                            const int buf = 2 * g + (acnt & 1), bph = (acnt >> 1) & 1;
+                            // a wait's verdict is made warp-uniform so that a timeout takes the whole warp out
+                            if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[buf], bph, abort_flag))) { ok = false; break; }
+                            tc_fence_after();
+                            float mc = 0.f, zc = 0.f;  // the running statistics of query tile qb (kept in registers)
 #pragma unroll
-                    for (int qb = 0; qb < kQTiles; ++qb) {
-                        if (qb >= nqt) continue;
-                        const SubBlock sb = sub_block(2 * (qt0 + qb) + my_row / kSub, sbq, n_sb, u.n_q);
-                        const int r = my_row % kSub;
-                        if (r < sb.valid) {
-                            const int64_t row = ((int64_t)u.l * mv.Hq + u.G * mv.hpg + sb.hh) * bv.total_q + u.q0 + sb.p0 + r;
-                            p.partial[(split * kGroups + g) * rows_total + row] = make_float2(m_raw[qb] * scale2, z[qb]);
+                            for (int k = 0; k < kQTiles; ++k)
+                                if (k == qb) {
+                                    mc = m_raw[k];
+                                    zc = z[k];
+                                }
+                            lse_accumulate(t_lane + buf * kRows, kt.valid, scale2, (live_mask >> qb) & 1u, mc, zc);
+#pragma unroll
+                            for (int k = 0; k < kQTiles; ++k)
+                                if (k == qb) {
+                                    m_raw[k] = mc;
+                                    z[k] = zc;
+                                }
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&acc_empty[buf]);
                         }
                     }
-                }
-            } else {
-                // stage the merged statistics of this chunk's rows, each warp for itself
-                float2 *sm = stats_sm + (warp - 2) * kQTiles * kRows;
-                for (int idx = lane; idx < nqt * kRows; idx += 32) {
-                    const int r = idx % kRows;
-                    const SubBlock sb = sub_block(2 * (qt0 + idx / kRows) + r / kSub, sbq, n_sb, u.n_q);
-                    float2 out = make_float2(0.f, 0.f);
-                    if (r % kSub < sb.valid)
-                        out = p.merged[((int64_t)u.l * mv.Hq + u.G * mv.hpg + sb.hh) * bv.total_q + u.q0 + sb.p0 + r % kSub];
-                    // rows 2k and 2k+1 share one float4: (-ref_2k, -ref_2k+1, w_2k, w_2k+1)
-                    float *smf = (float *)sm + (idx >> 1) * 4 + (idx & 1);
-                    smf[0] = out.x;
-                    smf[2] = out.y;
-                }
-                __syncwarp();
-                for (int t = t0 + g; t < t1 && ok; t += kGroups) {
-                    const KeyTile kt = key_tile(u, t);
-                    float c0 = 0.f, c1 = 0.f;
-#pragma unroll 1
-                    for (int qb = 0; qb < nqt && ok; ++qb, ++acnt) {
-                        const int buf = 2 * g + (acnt & 1), bph = (acnt >> 1) & 1;
-                        if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[buf], bph, abort_flag))) { ok = false; break; }
-                        tc_fence_after();
-                        const int v0 = sub_block(2 * (qt0 + qb), sbq, n_sb, u.n_q).valid;
-                        const int v1 = sub_block(2 * (qt0 + qb) + 1, sbq, n_sb, u.n_q).valid;
-                        colsum_accumulate(t_lane + buf * kRows, v0, v1, scale2, sm + qb * kRows, c0, c1);
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                    if (ok && t0 + g < t1) {
+#pragma unroll
+                        for (int qb = 0; qb < kQTiles; ++qb) {
+                            if (qb >= nqt) continue;
+                            const SubBlock sb = sub_block(2 * (qt0 + qb) + my_row / kSub, sbq, n_sb, u.n_q);
+                            const int r = my_row % kSub;
+                            if (r < sb.valid) {
+                                const int64_t row =
+                                    ((int64_t)u.l * mv.Hq + u.G * mv.hpg + sb.hh) * bv.total_q + u.q0 + sb.p0 + r;
+                                p.partial[(it.split * kGroups + g) * rows_total + row] =
+                                    make_float2(m_raw[qb] * scale2, z[qb]);
+                            }
+                        }
                     }
-                    if (ok && my_row < kt.valid) {
-                        float *dst = p.scores + ((int64_t)u.l * mv.G + u.G) * ((int64_t)bv.total_cache + bv.total_chunk) +
-                                     u.cache0 + u.chunk0 + kt.j0 + my_row;
-                        const float col = c0 + c1;
-                        *dst = c == 0 ? col : *dst + col;  // later query chunks add to the first chunk's sums
+                } else {
+                    // stage the merged statistics of this chunk's rows, each warp for itself (kept when the next
+                    // item has the same rows)
+                    float2 *sm = stats_sm + (warp - 2) * kQTiles * kRows;
+                    if (new_rows) {
+                        for (int idx = lane; idx < nqt * kRows; idx += 32) {
+                            const int r = idx % kRows;
+                            const SubBlock sb = sub_block(2 * (qt0 + idx / kRows) + r / kSub, sbq, n_sb, u.n_q);
+                            float2 out = make_float2(0.f, 0.f);
+                            if (r % kSub < sb.valid)
+                                out = p.merged[((int64_t)u.l * mv.Hq + u.G * mv.hpg + sb.hh) * bv.total_q + u.q0 + sb.p0 +
+                                               r % kSub];
+                            // rows 2k and 2k+1 share one float4: (-ref_2k, -ref_2k+1, w_2k, w_2k+1)
+                            float *smf = (float *)sm + (idx >> 1) * 4 + (idx & 1);
+                            smf[0] = out.x;
+                            smf[2] = out.y;
+                        }
+                        __syncwarp();
+                    }
+                    for (int t = t0 + g; t < t1 && ok; t += kGroups) {
+                        const KeyTile kt = key_tile(u, t);
+                        float c0 = 0.f, c1 = 0.f;
+#pragma unroll 1
+                        for (int qb = 0; qb < nqt && ok; ++qb, ++acnt) {
+                            const int buf = 2 * g + (acnt & 1), bph = (acnt >> 1) & 1;
+                            if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[buf], bph, abort_flag))) { ok = false; break; }
+                            tc_fence_after();
+                            const int v0 = sub_block(2 * (qt0 + qb), sbq, n_sb, u.n_q).valid;
+                            const int v1 = sub_block(2 * (qt0 + qb) + 1, sbq, n_sb, u.n_q).valid;
+                            colsum_accumulate(t_lane + buf * kRows, v0, v1, scale2, sm + qb * kRows, c0, c1);
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                        }
+                        if (ok && my_row < kt.valid) {
+                            float *dst = p.scores +
+                                         ((int64_t)u.l * mv.G + u.G) * ((int64_t)bv.total_cache + bv.total_chunk) +
+                                         u.cache0 + u.chunk0 + kt.j0 + my_row;
+                            const float col = c0 + c1;
+                            *dst = c == 0 ? col : *dst + col;  // later query chunks add to the first chunk's sums
+                        }
                     }
                 }
             }
@@ -605,7 +683,9 @@ cudaError_t launch_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensorMap &c
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(score_tc_kernel<kColsum, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    dim3 grid(p.splits, mv.L * mv.G, bv.batch);
+    p.n_items = p.splits * mv.L * mv.G * bv.batch;
+    const int sms = ctx.sm_count > 0 ? ctx.sm_count : 148;
+    dim3 grid(p.n_items < sms ? p.n_items : sms);  // persistent: one CTA per SM walks a contiguous range of items
     score_tc_kernel<kLse, D><<<grid, kTcThreads, smem, stream>>>(qm, cm, hm, p);
     dim3 mgrid((bv.max_q + 127) / 128, mv.L * mv.Hq, bv.batch);
     merge_stats_kernel<<<mgrid, 128, 0, stream>>>(p);
@@ -639,7 +719,7 @@ cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorVie
     if (!have_chunk) hm = cm;
     const int key_tiles = (bv.max_cache + kRows - 1) / kRows + (bv.max_chunk + kRows - 1) / kRows;
     const int max_splits = (int)min((size_t)kScoreMaxSplits, (partial_capacity / rows - 1) / kGroups);
-    TcParams p{mv, bv, partial, nullptr, row_lse, scores, ctx.d_status, min_q, 1, 2, 1};
+    TcParams p{mv, bv, partial, nullptr, row_lse, scores, ctx.d_status, min_q, 1, 2, 1, 0};
     p.splits = choose_splits(mv.L * mv.G * bv.batch, key_tiles, ctx.sm_count > 0 ? ctx.sm_count : 148, max_splits);
     p.merged = partial + (size_t)p.splits * kGroups * rows;
     return mv.d == 64 ? launch_d<64>(ctx, qm, cm, hm, p, stream) : launch_d<128>(ctx, qm, cm, hm, p, stream);
