@@ -29,6 +29,10 @@ from paper_2408_00167_b200 import workloads as wl  # noqa: E402
 METRIC = "candidate_kv_tokens_per_sec"
 UNIT = "tokens/s"
 FALLBACK_PEAK_GBS = 6650.0
+# DRAM bytes (read + write) of one full step from ncu, per configuration: captured on an 8-layer slice and scaled by
+# the unit count (profiles/step_kernels_c3_8layers.txt).  Must be set back to None whenever a kernel changes.
+TRAFFIC_BYTES = {"c3": 1002143744}
+MUFU_PER_CLK_PER_SM = 16   # exp2 results per clock per SM (4 per scheduler)
 
 
 def peak_hbm():
@@ -241,6 +245,11 @@ def run_ours(args, cfg: wl.Config):
     h2d = sum(host[k].numel() * host[k].element_size() for k in ("q", "chunk_k", "chunk_v", "chunk_pos"))
     d2h = kept_host.numel() * 4 + len_host.numel() * 4
     fb.finch_ctx_destroy(ctx)
+    sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
+    chunk_len = np.diff(st["chunk_off"]).astype(np.int64)
+    n_cand = st["cache_len"].astype(np.int64) + chunk_len
+    n_q = np.diff(st["q_off"]).astype(np.int64)
+    exps = float((n_cand * n_q).sum()) * cfg.n_layers * cfg.n_q_heads   # logits per sweep
     if rank != 0:
         return None
     peak, peak_kind = peak_hbm()
@@ -260,11 +269,17 @@ def run_ours(args, cfg: wl.Config):
                 "d2h_bytes_per_step": int(d2h), "ms_per_step": ms_e2e},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_kind": f"of {peak_kind}",
+                     "traffic": TRAFFIC_BYTES.get(cfg.name) if cfg.n_layers == wl.CONFIGS[cfg.name].n_layers else None,
+                     "peak_kind": f"of {peak_kind}",
                      "algorithmic_bytes_per_step": counts["contract_bytes"],
                      "kernel": "whole step (score + select + compact launches)"},
         "phases_ms": {"score": float(phase[0]), "select": float(phase[1]), "compact": float(phase[2])},
+        # the scoring phase is bound by the exponentials (two sweeps, one exp2 per logit each), not by HBM
+        "score_alu": {"bound": "alu", "unit": "Gexp2/s", "achieved": 2 * exps / (phase[0] * 1e-3) / 1e9,
+                      "peak": MUFU_PER_CLK_PER_SM * sm_count * (clocks.get("sm_mhz") or 1965) * 1e6 / 1e9,
+                      "note": "peak = 16 exp2/clk/SM x SMs x sampled SM clock"},
     }
+    line["score_alu"]["frac"] = line["score_alu"]["achieved"] / line["score_alu"]["peak"]
     return line
 
 
