@@ -143,7 +143,7 @@ def test_workspace_bytes_is_host_arithmetic(lib):
     try:
         b = _Fake.batch()
         n = fb.finch_workspace_bytes(ctx, b)
-        lse = 2 * 8 * 96 * 8 * 17
+        lse = 2 * 8 * 96 * 8 * 33
         scores = 2 * 2 * (256 + 512) * 4
         assert n >= lse + scores and n % 256 == 0
         bigger = _Fake.batch(total_q=192)
@@ -153,5 +153,34 @@ def test_workspace_bytes_is_host_arithmetic(lib):
         assert lib.finch_workspace_bytes(None, C.byref(b.c), C.byref(out)) == fb.FINCH_ERR_INVALID_ARG
         status = C.c_int32()
         assert lib.finch_device_status(ctx, None, C.byref(status)) == fb.FINCH_ERR_UNSUPPORTED
+    finally:
+        fb.finch_ctx_destroy(ctx)
+
+
+def test_step_host_validation(lib):
+    """finch_step_host checks its staging tensors and host pointers before anything is copied."""
+    ctx = fb.finch_ctx_create(**_cfg())
+    try:
+        b = _Fake.batch()
+        c = b.c
+        host = _Fake.base + 0xB000_0000
+
+        def call(stage_q=None, host_q=host, host_len=host + 0x100_0000, ws_bytes=1 << 30):
+            sq = stage_q or _Fake.tensor(0, c.total_q, heads=8)
+            sk, sv = _Fake.tensor(3, c.total_chunk), _Fake.tensor(4, c.total_chunk)
+            ck, cv = _Fake.tensor(1, c.total_cache), _Fake.tensor(2, c.total_cache)
+            ok, ov = _Fake.tensor(5, c.total_cache), _Fake.tensor(6, c.total_cache)
+            p = lambda x: C.c_void_p(x)
+            return lib.finch_step_host(ctx, p(host_q), p(host + 0x10_0000), p(host + 0x20_0000), p(host + 0x30_0000),
+                                       C.byref(sq), C.byref(sk), C.byref(sv), p(_Fake.base + 0xA300_0000), C.byref(ck),
+                                       C.byref(cv), p(_Fake.base + 0xA200_0000), C.byref(c), C.byref(ok), C.byref(ov),
+                                       p(_Fake.base + 0xA400_0000), p(_Fake.base + 0xA000_0000),
+                                       p(_Fake.base + 0xA100_0000), p(host + 0x40_0000), p(host_len),
+                                       p(_Fake.base + 0x9000_0000), C.c_size_t(ws_bytes), None)
+        assert call() == fb.FINCH_ERR_UNSUPPORTED                      # valid: stops at the launch stage
+        assert call(stage_q=_Fake.tensor(0, c.total_q, heads=8, stride_tok=128)) == fb.FINCH_ERR_BAD_LAYOUT
+        assert call(host_q=None) == fb.FINCH_ERR_INVALID_ARG
+        assert call(host_len=None) == fb.FINCH_ERR_INVALID_ARG
+        assert call(ws_bytes=1024) == fb.FINCH_ERR_WORKSPACE_TOO_SMALL
     finally:
         fb.finch_ctx_destroy(ctx)
