@@ -44,7 +44,7 @@ finch_status check_batch(const finch_ctx *ctx, const finch_batch *b) {
 }
 
 struct WsLayout {
-    size_t lse_off, lse_bytes;        // softmax statistics: one float2 per prompt row and key split
+    size_t lse_off, lse_bytes;        // scoring scratch: row statistics per key split and group, partial scores
     size_t scores_off, scores_bytes;  // scores inside finch_step when the caller gives none
     size_t total;
 };
@@ -53,7 +53,9 @@ WsLayout ws_layout(const finch_ctx *ctx, const finch_batch *b) {
     WsLayout w{};
     const ModelView &mv = ctx->model;
     w.lse_off = 0;
-    w.lse_bytes = align_up((size_t)mv.L * mv.Hq * (size_t)b->total_q * sizeof(float2) * (kScoreMaxSplits * 4 + 1));
+    const size_t n_scores = (size_t)mv.L * mv.G * ((size_t)b->total_cache + b->total_chunk);
+    w.lse_bytes = align_up((size_t)mv.L * mv.Hq * (size_t)b->total_q * sizeof(float2) * (kScoreMaxSplits * 4 + 1) +
+                           (4 * n_scores + 2) * sizeof(float));  // row statistics, then per-group partial scores
     w.scores_off = w.lse_off + w.lse_bytes;
     w.scores_bytes = align_up((size_t)mv.L * mv.G * ((size_t)b->total_cache + b->total_chunk) * sizeof(float));
     w.total = w.scores_off + w.scores_bytes;

@@ -10,10 +10,12 @@
 //   kColsum  D = Ktile x Qtile^T: one key per lane, so the sum over prompt rows of exp2(s - max) / sum is a private
 //            running sum per thread -> scores.  Its prologue merges the splits' partial statistics (fixed order).
 //
-// Warp roles (320 threads): warp 0 lane 0 issues TMA loads (128-byte swizzle), warp 1 owns tensor memory and its
-// lane 0 issues tcgen05.mma (128 x 128 x 16, fp32 accumulate), warps 2-9 form two softmax groups of four warps.
-// The groups take alternate key tiles and each has its own pair of 128-column accumulators, so no sum ever crosses
-// threads and every scheduler has two softmax warps to hide tcgen05.ld and MUFU latency.  mbarriers connect the
+// Warp roles (576 threads): warp 0 lane 0 issues TMA loads (128-byte swizzle), warp 1 owns tensor memory and its
+// lane 0 issues tcgen05.mma (128 x 128 x 16, fp32 accumulate), warps 2-17 form four softmax groups of four warps.
+// Accumulators (key tile x query tile) are dealt to the groups round-robin, each group owning one 128-column
+// accumulator: every scheduler then has four softmax warps, enough to keep the MUFU unit busy while one of them
+// waits for its next accumulator.  Sums never cross threads: the first sweep keeps per-group partial statistics,
+// the second writes per-group partial column sums that a small kernel adds in a fixed order.  mbarriers connect the
 // roles; every wait is bounded and raises FINCH_DEV_TIMEOUT instead of hanging.  Candidate tiles never straddle the cache/chunk
 // boundary: the cache's rows are tiled first, then the chunk's.
 #include <limits.h>
@@ -29,12 +31,12 @@ using namespace ptx;
 constexpr int kRows = 128;       // rows per operand tile = MMA M = MMA N
 constexpr int kSub = 64;         // prompt rows per sub-block (two per query tile)
 constexpr int kQTiles = 4;       // query tiles resident at a time
-constexpr int kGroups = 2;       // softmax groups (four warps each); group g takes the split's key tiles g, g+2, ..
-constexpr int kAccBufs = 4;      // accumulators of 128 fp32 columns in tensor memory (all 512 columns), two per group
+constexpr int kGroups = 4;       // softmax groups (four warps each); accumulator number A goes to group A % 4
+constexpr int kAccBufs = 4;      // accumulators of 128 fp32 columns in tensor memory (all 512 columns), one per group
 constexpr int kMaxStages = 4;    // key-tile ring
 constexpr int kTcThreads = 64 + kGroups * 128;
 constexpr int kSlabBytes = kRows * 128;                 // a 64-element (128-byte) wide slab of a 128-row tile
-constexpr int kStatsBytes = kGroups * 4 * kQTiles * kRows * 8;  // per softmax warp: (-max, 1/sum) of resident rows
+constexpr int kStatsBytes = 2 * kQTiles * kRows * 8;  // (-ref, weight) of the resident rows, double-buffered
 constexpr int kAuxBytes = 1024 + kStatsBytes;
 constexpr int kSmemLimit = 232448;                      // 227 KiB per CTA
 
@@ -47,6 +49,7 @@ struct TcParams {
     float2 *merged;    // [L][Hq][total_q] (-reference, weight) per prompt row after merging the parts
     float *row_lse;    // nullable
     float *scores;
+    float *score_parts;  // [kGroups][L][G][total_cand] per-group partial column sums
     int *status;
     int min_q;         // requests with fewer prompt rows are left to the warp-level path
     int splits;        // key splits per unit (grid x)
@@ -169,18 +172,15 @@ __device__ __forceinline__ void lse_chunk(const uint32_t (&r)[32], int nv, float
 // loads but skip the arithmetic, whose input would be whatever the shared memory held before.
 __device__ __forceinline__ void lse_accumulate(uint32_t taddr, int valid, float scale2, bool live, float &m_raw,
                                                float &z) {
-    uint32_t r[2][32];
-    __syncwarp();
-    tmem_ld_x32_issue(taddr, r[0]);
-#pragma unroll
-    for (int cc = 0; cc < 4; ++cc) {
-        if (cc * 32 >= valid) break;
-        tmem_ld_x32_wait(r[cc & 1]);
-        if ((cc + 1) * 32 < valid) {  // start the next chunk's load before working on this one
-            __syncwarp();
-            tmem_ld_x32_issue(taddr + (cc + 1) * 32, r[(cc + 1) & 1]);
-        }
-        if (live) lse_chunk(r[cc & 1], valid - cc * 32, scale2, m_raw, z);
+    // one 32-column chunk at a time: with four softmax warps per scheduler the other warps cover the tensor-memory
+    // latency, and a single register buffer keeps the kernel inside its register budget
+#pragma unroll 1
+    for (int cc = 0; cc * 32 < valid; ++cc) {
+        uint32_t r[32];
+        __syncwarp();
+        tmem_ld_x32_issue(taddr + cc * 32, r);
+        tmem_ld_x32_wait(r);
+        if (live) lse_chunk(r, valid - cc * 32, scale2, m_raw, z);
     }
 }
 
@@ -211,20 +211,15 @@ __device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[32], int nv, fl
 __device__ __forceinline__ void colsum_accumulate(uint32_t taddr, int v0, int v1, float scale2, const float2 *sm,
                                                   float &c0, float &c1) {
     const float4 *sm4 = (const float4 *)sm;
-    uint32_t r[2][32];
     // chunks 0 and 1 cover the tile's first 64-row half (always present), chunks 2 and 3 the second half
     const int last = v1 > 0 ? 4 : 2;
-    __syncwarp();
-    tmem_ld_x32_issue(taddr, r[0]);
-#pragma unroll
-    for (int cc = 0; cc < 4; ++cc) {
-        if (cc >= last) break;
-        tmem_ld_x32_wait(r[cc & 1]);
-        if (cc + 1 < last) {  // start the next chunk's load before working on this one
-            __syncwarp();
-            tmem_ld_x32_issue(taddr + (cc + 1) * 32, r[(cc + 1) & 1]);
-        }
-        colsum_chunk(r[cc & 1], (cc < 2 ? v0 : v1) - (cc & 1) * 32, scale2, sm4 + cc * 16, c0, c1);
+#pragma unroll 1
+    for (int cc = 0; cc < last; ++cc) {
+        uint32_t r[32];
+        __syncwarp();
+        tmem_ld_x32_issue(taddr + cc * 32, r);
+        tmem_ld_x32_wait(r);
+        colsum_chunk(r, (cc < 2 ? v0 : v1) - (cc & 1) * 32, scale2, sm4 + cc * 16, c0, c1);
     }
 }
 
@@ -280,9 +275,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     uint64_t *empty = full + kMaxStages;
     uint64_t *acc_full = empty + kMaxStages;
     uint64_t *acc_empty = acc_full + kAccBufs;
-    uint32_t *tmem_slot = (uint32_t *)(acc_empty + kAccBufs);
+    uint64_t *stats_ready = acc_empty + kAccBufs;  // all softmax warps have staged their share of the statistics
+    uint32_t *tmem_slot = (uint32_t *)(stats_ready + 1);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
-    float2 *stats_sm = (float2 *)(aux + 1024);  // [8 softmax warps][q_tiles * 128] row statistics, kColsum only
+    float2 *stats_sm = (float2 *)(aux + 1024);  // [2][q_tiles * 128] row statistics, kColsum only
 
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
@@ -300,8 +296,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         }
         for (int b = 0; b < kAccBufs; ++b) {
             mbar_init(&acc_full[b], 1);
-            mbar_init(&acc_empty[b], 4);  // one arrival per softmax warp
+            mbar_init(&acc_empty[b], 4);  // one arrival per softmax warp of the owning group
         }
+        mbar_init(stats_ready, 4 * kGroups);
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -377,47 +374,30 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_bf16_f32(kRows, kRows);
             const uint64_t q_desc = smem_desc_sw128(smem_u32(q_res)), ring_desc = smem_desc_sw128(smem_u32(k_ring));
-            // The two softmax groups consume independent streams of accumulators (group g: key tiles t0 + g,
-            // t0 + g + 2, .. of the split, every resident query tile of each).  The issuer serves whichever group
-            // has a free accumulator and a loaded key tile, so neither group waits for the other's backlog.
+            // Accumulators are issued in order (item, key tile, query tile); number A lands in buffer A % 4, which
+            // belongs to softmax group A % 4.  With equal work per accumulator the groups free their buffers in the
+            // same rotation, so in-order issue does not starve anyone.
             bool ok = true;
-            int kn = 0, qcnt = 0, q_key = -1;
-            int acnt[kGroups] = {0, 0};
+            int A = 0, qcnt = 0, q_key = -1, st = 0, sph = 0;
             for (int w = w0; w < w1 && ok; ++w) {
                 const Item it = decode_item(p, w, false);
                 if (!it.run) continue;
-                const int n_t = it.t1 - it.t0;
-                for (int c = 0; c < it.n_chunks && ok; ++c, kn += n_t) {
+                for (int c = 0; c < it.n_chunks && ok; ++c) {
                     const int nqt = min(p.q_tiles, it.n_qt - c * p.q_tiles);
                     if (!(it.n_chunks == 1 && q_key == it.key)) {
                         if (!mbar_wait(q_full, qcnt & 1, abort_flag)) { ok = false; break; }
                         ++qcnt;
                         q_key = it.n_chunks == 1 ? it.key : -1;
                     }
-                    int ti[kGroups] = {0, 1};  // next key tile (index within the split) of each group
-                    int qb[kGroups] = {0, 0};  // next query tile of that key tile
-                    // ring stage and phase of each group's next key tile, kept incrementally: this lone thread
-                    // cannot afford an integer division per poll
-                    int st[kGroups], sph[kGroups];
-#pragma unroll
-                    for (int g = 0; g < kGroups; ++g) {
-                        st[g] = (kn + g) % p.stages;
-                        sph[g] = ((kn + g) / p.stages) & 1;
-                    }
-                    uint32_t idle = 0;
-                    while ((ti[0] < n_t || ti[1] < n_t) && ok) {
-                        bool progressed = false;
-#pragma unroll
-                        for (int g = 0; g < kGroups; ++g) {
-                            if (ti[g] >= n_t) continue;
-                            const int stage = st[g];
-                            const int buf = 2 * g + (acnt[g] & 1), bph = (acnt[g] >> 1) & 1;
-                            if (!mbar_test_wait(&full[stage], sph[g]) || !mbar_test_wait(&acc_empty[buf], bph ^ 1))
-                                continue;
+                    for (int t = it.t0; t < it.t1 && ok; ++t) {
+                        if (!mbar_wait(&full[st], sph, abort_flag)) { ok = false; break; }
+                        const uint64_t kd = ring_desc + (uint64_t)((st * kTileBytes) >> 4);
+                        for (int qb = 0; qb < nqt; ++qb, ++A) {
+                            const int buf = A & 3;
+                            if (!mbar_wait(&acc_empty[buf], ((A >> 2) & 1) ^ 1, abort_flag)) { ok = false; break; }
                             tc_fence_after();
                             // one descriptor per operand tile; the K = 16 steps only advance its address field
-                            const uint64_t qd = q_desc + (uint64_t)((qb[g] * kTileBytes) >> 4);
-                            const uint64_t kd = ring_desc + (uint64_t)((stage * kTileBytes) >> 4);
+                            const uint64_t qd = q_desc + (uint64_t)((qb * kTileBytes) >> 4);
                             const uint64_t a_desc = MODE == kLse ? qd : kd, b_desc = MODE == kLse ? kd : qd;
                             const uint32_t d_addr = tmem_base + buf * kRows;
 #pragma unroll
@@ -429,27 +409,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                                     umma_bf16_acc(d_addr, a_desc + off, b_desc + off, idesc);
                             }
                             umma_commit(&acc_full[buf]);  // the accumulator is ready for its softmax group
-                            ++acnt[g];
-                            if (++qb[g] == nqt) {
-                                umma_commit(&empty[stage]);  // the stage may be refilled once these MMAs have read it
-                                qb[g] = 0;
-                                ti[g] += kGroups;
-                                st[g] += kGroups;
-                                while (st[g] >= p.stages) {
-                                    st[g] -= p.stages;
-                                    sph[g] ^= 1;
-                                }
-                            }
-                            progressed = true;
                         }
-                        if (progressed) {
-                            idle = 0;
-                        } else if ((++idle & 1023u) == 0) {  // keep polling; look at the abort flag now and then
-                            if (*abort_flag || idle > kSpinLimit) {
-                                *abort_flag = 1;
-                                ok = false;
-                            }
-                            if (idle > (1u << 16)) __nanosleep(64);
+                        if (ok) umma_commit(&empty[st]);  // the stage may be refilled once these MMAs have read it
+                        if (++st == p.stages) {
+                            st = 0;
+                            sph ^= 1;
                         }
                     }
                 }
@@ -458,11 +422,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     } else {
         // =================================================================== softmax warps (one TMEM lane per thread)
         const int quarter = warp & 3;            // tcgen05.ld reaches lanes 32 * (warp % 4) ..
-        const int g = (warp - 2) >> 2;           // softmax group: key tiles t0 + g, t0 + g + 2, ..
+        const int sw = warp - 2;                 // softmax warp 0..15
+        const int g = sw >> 2;                   // softmax group = the accumulator buffer it owns
         const int my_row = quarter * 32 + lane;  // row of the A tile this thread owns
-        const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + g * kRows;
         const float scale2 = mv.scale * kLog2e;
-        int acnt = 0, q_key = -1;
+        int A = 0, mine = 0, q_key = -1, epoch = 0;  // mine = accumulators this group has consumed (barrier phase)
         bool ok = true;
         for (int w = w0; w < w1 && ok; ++w) {
             const Item it = decode_item(p, w, false);
@@ -484,13 +449,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                         if (k < nqt && my_row % kSub < sub_block(2 * (qt0 + k) + my_row / kSub, sbq, n_sb, u.n_q).valid)
                             live_mask |= 1u << k;
                     }
-                    for (int t = t0 + g; t < t1 && ok; t += kGroups) {
+                    for (int t = t0; t < t1 && ok; ++t) {
                         const KeyTile kt = key_tile(u, t);
 #pragma unroll 1
-                        for (int qb = 0; qb < nqt && ok; ++qb, ++acnt) {
-                            const int buf = 2 * g + (acnt & 1), bph = (acnt >> 1) & 1;
+                        for (int qb = 0; qb < nqt && ok; ++qb, ++A) {
+                            if ((A & 3) != g) continue;  // another group's accumulator
                             // a wait's verdict is made warp-uniform so that a timeout takes the whole warp out
-                            if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[buf], bph, abort_flag))) { ok = false; break; }
+                            if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[g], mine & 1, abort_flag))) { ok = false; break; }
+                            ++mine;
                             tc_fence_after();
                             float mc = 0.f, zc = 0.f;  // the running statistics of query tile qb (kept in registers)
 #pragma unroll
@@ -499,7 +465,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                                     mc = m_raw[k];
                                     zc = z[k];
                                 }
-                            lse_accumulate(t_lane + buf * kRows, kt.valid, scale2, (live_mask >> qb) & 1u, mc, zc);
+                            lse_accumulate(t_acc, kt.valid, scale2, (live_mask >> qb) & 1u, mc, zc);
 #pragma unroll
                             for (int k = 0; k < kQTiles; ++k)
                                 if (k == qb) {
@@ -508,10 +474,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                                 }
                             tc_fence_before();
                             __syncwarp();
-                            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                            if (lane == 0) mbar_arrive(&acc_empty[g]);
                         }
                     }
-                    if (ok && t0 + g < t1) {
+                    if (ok) {  // every group reports every row of the chunk: (-inf, 0) where it saw no accumulator
 #pragma unroll
                         for (int qb = 0; qb < kQTiles; ++qb) {
                             if (qb >= nqt) continue;
@@ -526,11 +492,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                         }
                     }
                 } else {
-                    // stage the merged statistics of this chunk's rows, each warp for itself (kept when the next
-                    // item has the same rows)
-                    float2 *sm = stats_sm + (warp - 2) * kQTiles * kRows;
+                    // The merged statistics of the resident rows are staged once per CTA, every softmax warp its
+                    // share, into one of two buffers; a warp that has passed the barrier of epoch e has seen all
+                    // warps finish epoch e - 1, so the buffer of epoch e + 1 (= that of e - 1) is free by then.
                     if (new_rows) {
-                        for (int idx = lane; idx < nqt * kRows; idx += 32) {
+                        float2 *dst = stats_sm + (epoch & 1) * kQTiles * kRows;
+                        for (int idx = sw * 32 + lane; idx < nqt * kRows; idx += 16 * 32) {
                             const int r = idx % kRows;
                             const SubBlock sb = sub_block(2 * (qt0 + idx / kRows) + r / kSub, sbq, n_sb, u.n_q);
                             float2 out = make_float2(0.f, 0.f);
@@ -538,31 +505,37 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                                 out = p.merged[((int64_t)u.l * mv.Hq + u.G * mv.hpg + sb.hh) * bv.total_q + u.q0 + sb.p0 +
                                                r % kSub];
                             // rows 2k and 2k+1 share one float4: (-ref_2k, -ref_2k+1, w_2k, w_2k+1)
-                            float *smf = (float *)sm + (idx >> 1) * 4 + (idx & 1);
+                            float *smf = (float *)dst + (idx >> 1) * 4 + (idx & 1);
                             smf[0] = out.x;
                             smf[2] = out.y;
                         }
                         __syncwarp();
+                        if (lane == 0) mbar_arrive(stats_ready);
+                        if (!__all_sync(0xffffffffu, mbar_wait(stats_ready, epoch & 1, abort_flag))) { ok = false; break; }
+                        ++epoch;
                     }
-                    for (int t = t0 + g; t < t1 && ok; t += kGroups) {
+                    const float2 *sm = stats_sm + ((epoch - 1) & 1) * kQTiles * kRows;
+                    float *part = p.score_parts + ((int64_t)g * mv.L * mv.G + (int64_t)u.l * mv.G + u.G) *
+                                                      ((int64_t)bv.total_cache + bv.total_chunk) +
+                                  u.cache0 + u.chunk0;
+                    for (int t = t0; t < t1 && ok; ++t) {
                         const KeyTile kt = key_tile(u, t);
                         float c0 = 0.f, c1 = 0.f;
 #pragma unroll 1
-                        for (int qb = 0; qb < nqt && ok; ++qb, ++acnt) {
-                            const int buf = 2 * g + (acnt & 1), bph = (acnt >> 1) & 1;
-                            if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[buf], bph, abort_flag))) { ok = false; break; }
+                        for (int qb = 0; qb < nqt && ok; ++qb, ++A) {
+                            if ((A & 3) != g) continue;
+                            if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[g], mine & 1, abort_flag))) { ok = false; break; }
+                            ++mine;
                             tc_fence_after();
                             const int v0 = sub_block(2 * (qt0 + qb), sbq, n_sb, u.n_q).valid;
                             const int v1 = sub_block(2 * (qt0 + qb) + 1, sbq, n_sb, u.n_q).valid;
-                            colsum_accumulate(t_lane + buf * kRows, v0, v1, scale2, sm + qb * kRows, c0, c1);
+                            colsum_accumulate(t_acc, v0, v1, scale2, sm + qb * kRows, c0, c1);
                             tc_fence_before();
                             __syncwarp();
-                            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                            if (lane == 0) mbar_arrive(&acc_empty[g]);
                         }
-                        if (ok && my_row < kt.valid) {
-                            float *dst = p.scores +
-                                         ((int64_t)u.l * mv.G + u.G) * ((int64_t)bv.total_cache + bv.total_chunk) +
-                                         u.cache0 + u.chunk0 + kt.j0 + my_row;
+                        if (ok && my_row < kt.valid) {  // this group's share of the key's score (0 if it had none)
+                            float *dst = part + kt.j0 + my_row;
                             const float col = c0 + c1;
                             *dst = c == 0 ? col : *dst + col;  // later query chunks add to the first chunk's sums
                         }
@@ -603,9 +576,9 @@ merge_stats_kernel(TcParams p) {
     const int64_t row = ((int64_t)l * mv.Hq + h) * bv.total_q + u.q0 + pr;
     float M = -INFINITY, Z = 0.f;
     for (int s = 0; s * tps < k_tiles; ++s) {
-        const int parts = min(kGroups, min(k_tiles, (s + 1) * tps) - s * tps);
-        for (int g = 0; g < parts; ++g) {
+        for (int g = 0; g < kGroups; ++g) {
             const float2 pm = p.partial[(s * kGroups + g) * rows_total + row];
+            if (!(pm.y > 0.f)) continue;  // a group that saw none of this row's accumulators in this split
             const float nm = fmaxf(M, pm.x);
             Z = Z * ex2(M - nm) + pm.y * ex2(pm.x - nm);
             M = nm;
@@ -614,6 +587,24 @@ merge_stats_kernel(TcParams p) {
     const int k = ilogbf(Z);
     p.merged[row] = make_float2(-(M + (float)k), ldexpf(1.0f, k) / Z);
     if (p.row_lse) p.row_lse[row] = (M + log2f(Z)) * kLn2;
+}
+
+// scores = the four groups' partial column sums, added in group order.
+__global__ void __launch_bounds__(256)
+combine_scores_kernel(TcParams p) {
+    const ModelView &mv = p.mv;
+    const BatchView &bv = p.bv;
+    const UnitInfo u = unit_info(mv, bv, blockIdx.y, blockIdx.z);
+    if (!u.ok || u.n_q < p.min_q) return;
+    const int j = blockIdx.x * 256 + threadIdx.x;
+    if (j >= u.N) return;
+    const int64_t cand = (int64_t)bv.total_cache + bv.total_chunk;
+    const int64_t off = ((int64_t)u.l * mv.G + u.G) * cand + u.cache0 + u.chunk0 + j;
+    const int64_t gstride = (int64_t)mv.L * mv.G * cand;
+    float s = p.score_parts[off];
+#pragma unroll
+    for (int g = 1; g < kGroups; ++g) s += p.score_parts[g * gstride + off];
+    p.scores[off] = s;
 }
 
 // ------------------------------------------------------------------------------------------------ host side
@@ -690,7 +681,9 @@ cudaError_t launch_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensorMap &c
     dim3 mgrid((bv.max_q + 127) / 128, mv.L * mv.Hq, bv.batch);
     merge_stats_kernel<<<mgrid, 128, 0, stream>>>(p);
     score_tc_kernel<kColsum, D><<<grid, kTcThreads, smem, stream>>>(qm, cm, hm, p);
-    ctx.launches += 3;
+    dim3 cgrid((bv.max_cache + bv.max_chunk + 255) / 256, mv.L * mv.G, bv.batch);
+    combine_scores_kernel<<<cgrid, 256, 0, stream>>>(p);
+    ctx.launches += 4;
     return cudaGetLastError();
 }
 
@@ -701,7 +694,7 @@ bool score_tc_supported(const Ctx &ctx) {
 }
 
 // `partial` holds partial_capacity float2 entries; the key-split count is limited so that one entry per prompt
-// row, split and softmax group, plus one merged entry per row, fits.  Returns cudaErrorNotSupported (and launches nothing) when the tensors cannot be described
+// row, split and softmax group, one merged entry per row and the per-group partial scores fit.  Returns cudaErrorNotSupported (and launches nothing) when the tensors cannot be described
 // to the TMA unit; the caller then uses the warp-level path for every request.
 cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
                             const BatchView &bv, float *scores, float2 *partial, size_t partial_capacity,
@@ -709,7 +702,10 @@ cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorVie
     const ModelView &mv = ctx.model;
     if (mv.L * mv.G == 0 || bv.batch == 0 || bv.max_q == 0 || bv.max_cache + bv.max_chunk == 0) return cudaSuccess;
     const size_t rows = (size_t)mv.L * mv.Hq * (size_t)bv.total_q;
-    if (rows == 0 || partial_capacity < rows * (kGroups + 1)) return cudaErrorNotSupported;
+    // scratch layout (float2 units): per-split, per-group row statistics | merged row statistics | per-group scores
+    const size_t cand = (size_t)mv.L * mv.G * ((size_t)bv.total_cache + bv.total_chunk);
+    const size_t parts_f2 = (kGroups * cand + 1) / 2;
+    if (rows == 0 || partial_capacity < rows * (kGroups + 1) + parts_f2) return cudaErrorNotSupported;
     CUtensorMap qm, cm, hm;
     if (!make_map(&qm, q, mv.d, bv.total_q, mv.Hq, mv.L, kSub)) return cudaErrorNotSupported;
     const bool have_cache = bv.max_cache > 0, have_chunk = bv.max_chunk > 0;
@@ -718,10 +714,11 @@ cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorVie
     if (!have_cache) cm = hm;  // never dereferenced: no request has cache tiles
     if (!have_chunk) hm = cm;
     const int key_tiles = (bv.max_cache + kRows - 1) / kRows + (bv.max_chunk + kRows - 1) / kRows;
-    const int max_splits = (int)min((size_t)kScoreMaxSplits, (partial_capacity / rows - 1) / kGroups);
-    TcParams p{mv, bv, partial, nullptr, row_lse, scores, ctx.d_status, min_q, 1, 2, 1, 0};
+    const int max_splits = (int)min((size_t)kScoreMaxSplits, ((partial_capacity - parts_f2) / rows - 1) / kGroups);
+    TcParams p{mv, bv, partial, nullptr, row_lse, scores, nullptr, ctx.d_status, min_q, 1, 2, 1, 0};
     p.splits = choose_splits(mv.L * mv.G * bv.batch, key_tiles, ctx.sm_count > 0 ? ctx.sm_count : 148, max_splits);
     p.merged = partial + (size_t)p.splits * kGroups * rows;
+    p.score_parts = (float *)(p.merged + rows);
     return mv.d == 64 ? launch_d<64>(ctx, qm, cm, hm, p, stream) : launch_d<128>(ctx, qm, cm, hm, p, stream);
 }
 

@@ -143,7 +143,7 @@ def test_workspace_bytes_is_host_arithmetic(lib):
     try:
         b = _Fake.batch()
         n = fb.finch_workspace_bytes(ctx, b)
-        lse = 2 * 8 * 96 * 8 * 33
+        lse = 2 * 8 * 96 * 8 * 33 + 4 * 2 * 2 * (256 + 512) * 4
         scores = 2 * 2 * (256 + 512) * 4
         assert n >= lse + scores and n % 256 == 0
         bigger = _Fake.batch(total_q=192)
