@@ -109,24 +109,17 @@ finch_status validate_compact(const finch_ctx *ctx, const int32_t *kept_idx, con
 
 namespace finch {
 
-// Tensor cores take the requests whose prompt has at least 64 rows (bf16, supported head_dim); warp-level dot
-// products take the rest.  batch.min_q lets the host skip the launch that would find no request of its class.
+// Tensor cores take every request when the context allows them (bf16, supported head_dim, one KV head per group);
+// warp-level dot products take everything else, and also a batch whose tensors the TMA unit cannot describe.
 cudaError_t run_score(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
                       const BatchView &bv, float *scores, float2 *scratch, size_t scratch_capacity, float *row_lse,
                       cudaStream_t stream) {
-    constexpr int kTensorCoreMinRows = 64;
-    int simt_below = INT_MAX;
-    if (score_tc_supported(ctx) && bv.max_q >= kTensorCoreMinRows) {
+    if (score_tc_supported(ctx)) {
         const cudaError_t e = launch_score_tc(ctx, q, cache_k, chunk_k, bv, scores, scratch, scratch_capacity, row_lse,
-                                              kTensorCoreMinRows, stream);
-        if (e == cudaSuccess) {
-            if (bv.min_q >= kTensorCoreMinRows) return cudaSuccess;
-            simt_below = kTensorCoreMinRows;
-        } else if (e != cudaErrorNotSupported) {
-            return e;
-        }
+                                              /*min_q=*/1, stream);
+        if (e != cudaErrorNotSupported) return e;
     }
-    return launch_score_simt(ctx, q, cache_k, chunk_k, bv, scores, scratch, row_lse, simt_below, stream);
+    return launch_score_simt(ctx, q, cache_k, chunk_k, bv, scores, scratch, row_lse, INT_MAX, stream);
 }
 
 }  // namespace finch

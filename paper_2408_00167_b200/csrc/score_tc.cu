@@ -1,4 +1,4 @@
-// Prompt-guided scoring on the 5th-generation tensor cores (bf16 inputs, prompts of at least 64 rows).
+// Prompt-guided scoring on the 5th-generation tensor cores (bf16 inputs, head_dim 64 or 128, one KV head per group).
 //
 // One kernel template, two sweeps over the logits S = Q K^T of a unit (layer, KV head, request).  A CTA owns one
 // split of the unit's 128-key tiles and keeps up to four 128-row tiles of the group's prompt queries resident in
@@ -127,8 +127,8 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
 // kLse: fold 32 columns (keys) of one accumulator row into the row's running (reference, sum of exp2).
 // The reference is the maximum of the row's first chunk, not the running maximum: any reference works as long as
 // the sum stays finite, and skipping the per-element maximum saves a quarter of the instructions.  If the sum
-// overflows (a later logit more than ~2^7 base-2 units above the reference) the reference is raised and the chunk
-// redone.  Columns at or beyond nv hold no key and count nothing.
+// overflows (a later logit more than ~2^7 base-2 units above the reference, or many nearly that far) the reference
+// moves up and the chunk is redone.  Columns at or beyond nv hold no key and count nothing.
 __device__ __forceinline__ void lse_chunk(const uint32_t (&r)[32], int nv, float scale2, float &m_raw, float &z) {
     float v[32];
 #pragma unroll
@@ -143,7 +143,7 @@ __device__ __forceinline__ void lse_chunk(const uint32_t (&r)[32], int nv, float
         for (int e = 1; e < 32; ++e) cmax = fmaxf(cmax, v[e]);
         m_raw = cmax;
     }
-    for (int attempt = 0; attempt < 8; ++attempt) {
+    for (int attempt = 0; attempt < 2; ++attempt) {
         const float negm = -(m_raw * scale2);
         const uint64_t s2 = pack2(scale2, scale2), n2 = pack2(negm, negm);
         uint64_t acc0 = 0, acc1 = 0;  // two pairs of partial sums (+0.0f bit patterns)
@@ -163,8 +163,19 @@ __device__ __forceinline__ void lse_chunk(const uint32_t (&r)[32], int nv, float
             z = zn;
             break;
         }
-        m_raw += 64.0f / scale2;  // overflow: lift the reference by 2^64 and rescale what has been summed so far
-        z *= 5.421010862427522e-20f;
+        // overflow: move the reference up and redo the chunk
+        float cmax = v[0];
+#pragma unroll
+        for (int e = 1; e < 32; ++e) cmax = fmaxf(cmax, v[e]);
+        // The new reference must cover the chunk's largest logit and what has been summed so far (z = 2^e * [1, 2)
+        // against the old reference, e from z's exponent field), so that the redone sum is at most 1 + 32.  The
+        // factor between the two references (the same rounded products the chunks subtract) is applied in two
+        // halves, since z may be near 2^127 while the factor is below the smallest normal number.
+        const float lift = (float)(((__float_as_int(z) >> 23) & 0xff) - 126);
+        const float m_new = fmaxf(cmax, fmaf(lift, __frcp_rn(scale2), m_raw));
+        const float half_d = 0.5f * (__fmul_rn(m_raw, scale2) - __fmul_rn(m_new, scale2));
+        z = (z * ex2(half_d)) * ex2(half_d);
+        m_raw = m_new;
     }
 }
 
@@ -579,8 +590,12 @@ merge_stats_kernel(TcParams p) {
         for (int g = 0; g < kGroups; ++g) {
             const float2 pm = p.partial[(s * kGroups + g) * rows_total + row];
             if (!(pm.y > 0.f)) continue;  // a group that saw none of this row's accumulators in this split
-            const float nm = fmaxf(M, pm.x);
-            Z = Z * ex2(M - nm) + pm.y * ex2(pm.x - nm);
+            // A part's sum can be as large as 2^127 against a reference that far below its largest logit: move
+            // the sum's exponent into the reference first, so that neither factor below leaves the fp32 range.
+            const int e = ilogbf(pm.y);
+            const float px = pm.x + (float)e, py = ldexpf(pm.y, -e);
+            const float nm = fmaxf(M, px);
+            Z = Z * ex2(M - nm) + py * ex2(px - nm);
             M = nm;
         }
     }

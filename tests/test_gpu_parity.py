@@ -56,7 +56,7 @@ SHAPES = [
     ("bf16", 8, 2, 128, [(16, 9999, 200, 100)]),
     ("bf16", 4, 4, 64, [(63, 9999, 129, 64)]),
     ("bf16", 8, 2, 128, [(5, 9999, 64, 17), (33, 9999, 100, 300), (20, 9999, 1, 1)]),
-    # tensor-core path (>= 64 prompt rows): partial row blocks, partial key tiles on both sides of the cache/chunk seam
+    # partial row blocks, partial key tiles on both sides of the cache/chunk seam
     ("bf16", 8, 2, 128, [(130, 9999, 300, 333)]),
     ("bf16", 4, 2, 64, [(64, 9999, 1, 129), (257, 9999, 257, 255), (40, 9999, 90, 70)]),
 ]
@@ -68,6 +68,26 @@ def test_small_shapes_with_ragged_tails(dtype, Hq, Hkv, d, reqs, group_mode):
     cfg = _small("c3", dtype, Hq, Hkv, d, reqs, group_mode=group_mode, planted_frac=0.03)
     st = wl.steady_state(cfg, [0, 1], step=3)
     _run_and_check(cfg, st, 2, parts=(group_mode == 1))
+
+
+@pytest.mark.parametrize("scale", [6.0, 40.0])
+def test_wide_logit_range_on_the_tensor_core_path(scale):
+    # logits spread over hundreds (scale 6) or thousands (scale 40) of binary orders: the row sums, taken against the
+    # maximum of the first 32 keys only, overflow in later chunks and have to move their reference
+    cfg = _small("c3", "bf16", 8, 2, 128, [(130, 9999, 300, 333), (20, 9999, 40, 250)], planted_frac=0.03)
+    st = wl.steady_state(cfg, [0, 1], step=2)
+    g = GpuStep(cfg, st, 2, scale=scale)
+    try:
+        g.run_parts()
+        assert g.status() == 0
+        res = g.results()
+        ref, ref_lse = oracle_scores(cfg, st, scale=scale, want_lse=True)
+        summary = check_parity(cfg, st, res, ref)
+        assert summary["max_rel_err"] < 1e-3
+        valid = ~np.isnan(res["row_lse"])
+        np.testing.assert_allclose(res["row_lse"][valid], ref_lse[valid], rtol=2e-6, atol=2e-4)
+    finally:
+        g.close()
 
 
 def test_row_lse_output_matches_oracle():
