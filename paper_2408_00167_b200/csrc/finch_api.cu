@@ -55,7 +55,8 @@ WsLayout ws_layout(const finch_ctx *ctx, const finch_batch *b) {
     w.lse_off = 0;
     const size_t n_scores = (size_t)mv.L * mv.G * ((size_t)b->total_cache + b->total_chunk);
     w.lse_bytes = align_up((size_t)mv.L * mv.Hq * (size_t)b->total_q * sizeof(float2) * (kScoreMaxSplits * 4 + 1) +
-                           (4 * n_scores + 2) * sizeof(float));  // row statistics, then per-group partial scores
+                           (4 * n_scores + 2) * sizeof(float) +  // row statistics, per-group partial scores,
+                           ((size_t)b->batch + 1) * 8 + 4096);   // and the item plan of a multi-request batch
     w.scores_off = w.lse_off + w.lse_bytes;
     w.scores_bytes = align_up((size_t)mv.L * mv.G * ((size_t)b->total_cache + b->total_chunk) * sizeof(float));
     w.total = w.scores_off + w.scores_bytes;

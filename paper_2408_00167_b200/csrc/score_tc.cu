@@ -32,6 +32,7 @@ constexpr int kRows = 128;       // rows per operand tile = MMA M = MMA N
 constexpr int kSub = 64;         // prompt rows per sub-block (two per query tile)
 constexpr int kQTiles = 4;       // query tiles resident at a time
 constexpr int kGroups = 4;       // softmax groups (four warps each); accumulator number A goes to group A % 4
+constexpr int kPlanBoundsInts = 1024;  // room for the per-CTA item bounds in the scratch (grid + 1 <= this)
 constexpr int kAccBufs = 4;      // accumulators of 128 fp32 columns in tensor memory (all 512 columns), one per group
 constexpr int kMaxStages = 4;    // key-tile ring
 constexpr int kTcThreads = 64 + kGroups * 128;
@@ -56,6 +57,8 @@ struct TcParams {
     int stages;        // key-tile ring depth that fits beside the resident queries
     int q_tiles;       // query tiles resident at a time (1..4), sized from the batch's longest prompt
     int n_items;       // work items = splits x units x requests, walked by a persistent grid
+    const int *bounds;              // [grid + 1] first item of every CTA (work-weighted), or null: equal item counts
+    unsigned long long *work_prefix;  // [batch + 1] accumulators of all items of the requests before b (plan scratch)
 };
 
 struct KeyTile {
@@ -294,8 +297,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
     // this CTA's contiguous range of work items
-    const int w0 = (int)((int64_t)blockIdx.x * p.n_items / gridDim.x);
-    const int w1 = (int)((int64_t)(blockIdx.x + 1) * p.n_items / gridDim.x);
+    const int w0 = p.bounds ? p.bounds[blockIdx.x] : (int)((int64_t)blockIdx.x * p.n_items / gridDim.x);
+    const int w1 = p.bounds ? p.bounds[blockIdx.x + 1] : (int)((int64_t)(blockIdx.x + 1) * p.n_items / gridDim.x);
     const int64_t rows_total = (int64_t)mv.L * mv.Hq * bv.total_q;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -569,6 +572,72 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     }
 }
 
+// With several requests in the batch the items differ in size (accumulators = key tiles x query tiles of their
+// request), so equal item counts per CTA would leave the grid waiting for the CTAs that drew the long prompts and
+// large caches.  This one-block kernel sums the work per request (items are ordered request-major, and all items
+// of a request cost about the same), then gives every CTA of the persistent grid a contiguous item range of about
+// equal work: bounds[i] = the item at which the running work passes i / n_ctas of the total.
+__global__ void __launch_bounds__(1024)
+plan_items_kernel(TcParams p, int *bounds, int n_ctas) {
+    __shared__ unsigned long long warp_sum[32];
+    __shared__ unsigned long long carry_s;
+    const ModelView &mv = p.mv;
+    const BatchView &bv = p.bv;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const unsigned long long ipr = (unsigned long long)mv.L * mv.G * p.splits;  // items per request
+    if (tid == 0) {
+        carry_s = 0;
+        p.work_prefix[0] = 0;
+    }
+    __syncthreads();
+    for (int base = 0; base < bv.batch; base += 1024) {
+        const int b = base + tid;
+        unsigned long long cost = 0;
+        if (b < bv.batch) {
+            const UnitInfo u = unit_info(mv, bv, 0, b);
+            if (u.ok && u.n_q >= p.min_q && u.N > 0) {
+                const int sb = mv.hpg * ((u.n_q + kSub - 1) / kSub);
+                // key tiles of one split x query tiles, plus a little for the item's fixed costs
+                cost = ipr * (unsigned long long)((n_key_tiles(u) + p.splits - 1) / p.splits * ((sb + 1) / 2) + 2);
+            }
+        }
+        unsigned long long incl = cost;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned long long up = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += up;
+        }
+        if (lane == 31) warp_sum[wid] = incl;
+        __syncthreads();
+        unsigned long long before = carry_s;
+        for (int w = 0; w < wid; ++w) before += warp_sum[w];
+        if (b < bv.batch) p.work_prefix[b + 1] = before + incl;
+        __syncthreads();
+        if (tid == 1023) carry_s = before + incl;
+        __syncthreads();
+    }
+    const unsigned long long total = carry_s;
+    for (int i = tid; i <= n_ctas; i += 1024) {
+        int item;
+        if (i == 0) {
+            item = 0;
+        } else if (i == n_ctas || total == 0) {
+            item = p.n_items;
+        } else {
+            const unsigned long long target = total / n_ctas * i + total % n_ctas * i / n_ctas;
+            int lo = 0, hi = bv.batch - 1;  // the last request whose prefix is <= target
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (p.work_prefix[mid] <= target) lo = mid; else hi = mid - 1;
+            }
+            const unsigned long long span = p.work_prefix[lo + 1] - p.work_prefix[lo];
+            const unsigned long long into = span ? (target - p.work_prefix[lo]) * ipr / span : 0;
+            item = (int)((unsigned long long)lo * ipr + (into < ipr ? into : ipr));
+        }
+        bounds[i] = item;
+    }
+}
+
 // Merge the per-split, per-group partial statistics of every prompt row (fixed order) into the pair the column pass
 // uses: weights are exp2(s2 - R) * w with R = M + floor(log2 Z) and w = 2^floor(log2 Z) / Z in (1/2, 1], so the
 // exponent never exceeds a few units whatever reference the parts were summed against.
@@ -692,6 +761,12 @@ cudaError_t launch_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensorMap &c
     p.n_items = p.splits * mv.L * mv.G * bv.batch;
     const int sms = ctx.sm_count > 0 ? ctx.sm_count : 148;
     dim3 grid(p.n_items < sms ? p.n_items : sms);  // persistent: one CTA per SM walks a contiguous range of items
+    if (bv.batch > 1 && (int)grid.x < kPlanBoundsInts) {  // requests of different sizes: ranges of equal work
+        int *bounds = (int *)(p.work_prefix + bv.batch + 1);
+        plan_items_kernel<<<1, 1024, 0, stream>>>(p, bounds, (int)grid.x);
+        p.bounds = bounds;
+        ctx.launches += 1;
+    }
     score_tc_kernel<kLse, D><<<grid, kTcThreads, smem, stream>>>(qm, cm, hm, p);
     dim3 mgrid((bv.max_q + 127) / 128, mv.L * mv.Hq, bv.batch);
     merge_stats_kernel<<<mgrid, 128, 0, stream>>>(p);
@@ -717,10 +792,12 @@ cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorVie
     const ModelView &mv = ctx.model;
     if (mv.L * mv.G == 0 || bv.batch == 0 || bv.max_q == 0 || bv.max_cache + bv.max_chunk == 0) return cudaSuccess;
     const size_t rows = (size_t)mv.L * mv.Hq * (size_t)bv.total_q;
-    // scratch layout (float2 units): per-split, per-group row statistics | merged row statistics | per-group scores
+    // scratch layout (float2 units): per-split, per-group row statistics | merged row statistics | item plan |
+    // per-group scores
     const size_t cand = (size_t)mv.L * mv.G * ((size_t)bv.total_cache + bv.total_chunk);
     const size_t parts_f2 = (kGroups * cand + 1) / 2;
-    if (rows == 0 || partial_capacity < rows * (kGroups + 1) + parts_f2) return cudaErrorNotSupported;
+    const size_t plan_f2 = (size_t)bv.batch + 1 + kPlanBoundsInts / 2;  // 64-bit work prefix, then the CTA bounds
+    if (rows == 0 || partial_capacity < rows * (kGroups + 1) + parts_f2 + plan_f2) return cudaErrorNotSupported;
     CUtensorMap qm, cm, hm;
     if (!make_map(&qm, q, mv.d, bv.total_q, mv.Hq, mv.L, kSub)) return cudaErrorNotSupported;
     const bool have_cache = bv.max_cache > 0, have_chunk = bv.max_chunk > 0;
@@ -729,11 +806,13 @@ cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorVie
     if (!have_cache) cm = hm;  // never dereferenced: no request has cache tiles
     if (!have_chunk) hm = cm;
     const int key_tiles = (bv.max_cache + kRows - 1) / kRows + (bv.max_chunk + kRows - 1) / kRows;
-    const int max_splits = (int)min((size_t)kScoreMaxSplits, ((partial_capacity - parts_f2) / rows - 1) / kGroups);
-    TcParams p{mv, bv, partial, nullptr, row_lse, scores, nullptr, ctx.d_status, min_q, 1, 2, 1, 0};
+    const int max_splits =
+        (int)min((size_t)kScoreMaxSplits, ((partial_capacity - parts_f2 - plan_f2) / rows - 1) / kGroups);
+    TcParams p{mv, bv, partial, nullptr, row_lse, scores, nullptr, ctx.d_status, min_q, 1, 2, 1, 0, nullptr, nullptr};
     p.splits = choose_splits(mv.L * mv.G * bv.batch, key_tiles, ctx.sm_count > 0 ? ctx.sm_count : 148, max_splits);
     p.merged = partial + (size_t)p.splits * kGroups * rows;
-    p.score_parts = (float *)(p.merged + rows);
+    p.work_prefix = (unsigned long long *)(p.merged + rows);
+    p.score_parts = (float *)(p.merged + rows + plan_f2);
     return mv.d == 64 ? launch_d<64>(ctx, qm, cm, hm, p, stream) : launch_d<128>(ctx, qm, cm, hm, p, stream);
 }
 
