@@ -247,28 +247,72 @@ struct Item {
     bool run;
 };
 
-__device__ __forceinline__ Item decode_item(const TcParams &p, int w, bool report) {
-    Item it;
+// A role's position in its CTA's item range.  Items are walked in order, so the position (split, group, layer,
+// request) advances by counting, and everything that depends on the request alone (its batch metadata, tile counts)
+// is computed when the request changes: per item there is no division and no load from global memory.  A role
+// thread that stalls at every item boundary stalls the pipeline behind it.
+struct Walk {
+    int w, split, key, l, G, b;
+    UnitInfo req;  // metadata of request `req.b` (-1: none read yet); l and G are not kept here
+    int k_tiles, tps, sbq, n_sb, n_qt, n_chunks;
+    bool req_run;  // the request has prompt rows for this path and candidates
+};
+
+__device__ __forceinline__ void walk_init(Walk &k, const TcParams &p, int w0) {
     const int units = p.mv.L * p.mv.G;
-    it.split = w % p.splits;
-    it.key = w / p.splits;
-    it.u = unit_info(p.mv, p.bv, it.key % units, it.key / units);
-    it.run = false;
-    if (!it.u.ok) {
-        if (report) atomicOr(p.status, FINCH_DEV_BAD_BATCH);
-        return it;
+    k.w = w0;
+    k.split = w0 % p.splits;
+    k.key = w0 / p.splits;
+    const int unit = k.key % units;
+    k.b = k.key / units;
+    k.l = unit / p.mv.G;
+    k.G = unit % p.mv.G;
+    k.req.b = -1;
+}
+
+__device__ __forceinline__ void walk_next(Walk &k, const TcParams &p) {
+    ++k.w;
+    if (++k.split == p.splits) {
+        k.split = 0;
+        ++k.key;
+        if (++k.G == p.mv.G) {
+            k.G = 0;
+            if (++k.l == p.mv.L) {
+                k.l = 0;
+                ++k.b;
+            }
+        }
     }
-    if (it.u.n_q < p.min_q || it.u.N == 0) return it;
-    it.k_tiles = n_key_tiles(it.u);
-    it.tps = (it.k_tiles + p.splits - 1) / p.splits;  // key tiles per split
-    it.t0 = it.split * it.tps;
-    it.t1 = min(it.k_tiles, it.t0 + it.tps);
-    if (it.t0 >= it.t1) return it;
-    it.sbq = (it.u.n_q + kSub - 1) / kSub;  // sub-blocks per query head
-    it.n_sb = p.mv.hpg * it.sbq;
-    it.n_qt = (it.n_sb + 1) / 2;  // query tiles of the group
-    it.n_chunks = (it.n_qt + p.q_tiles - 1) / p.q_tiles;
-    it.run = true;
+}
+
+__device__ __forceinline__ Item walk_item(Walk &k, const TcParams &p, bool report) {
+    if (k.req.b != k.b) {
+        k.req = unit_info(p.mv, p.bv, 0, k.b);
+        const UnitInfo &u = k.req;
+        k.req_run = u.ok && u.n_q >= p.min_q && u.N > 0;
+        k.k_tiles = n_key_tiles(u);
+        k.tps = (k.k_tiles + p.splits - 1) / p.splits;  // key tiles per split
+        k.sbq = (u.n_q + kSub - 1) / kSub;              // sub-blocks per query head
+        k.n_sb = p.mv.hpg * k.sbq;
+        k.n_qt = (k.n_sb + 1) / 2;  // query tiles of the group
+        k.n_chunks = (k.n_qt + p.q_tiles - 1) / p.q_tiles;
+    }
+    Item it;
+    it.u = k.req;
+    it.u.l = k.l;
+    it.u.G = k.G;
+    it.key = k.key;
+    it.split = k.split;
+    it.k_tiles = k.k_tiles;
+    it.tps = k.tps;
+    it.sbq = k.sbq;
+    it.n_sb = k.n_sb;
+    it.n_qt = k.n_qt;
+    it.n_chunks = k.n_chunks;
+    it.t0 = k.split * k.tps;
+    it.t1 = min(k.k_tiles, it.t0 + k.tps);
+    it.run = k.req_run && it.t0 < it.t1;
+    if (!k.req.ok && report) atomicOr(p.status, FINCH_DEV_BAD_BATCH);
     return it;
 }
 
@@ -335,8 +379,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             prefetch_tensormap(&chunk_map);
             int kcnt = 0, qcnt = 0, pst = 0, pph = 0, last_stage = 0, last_ph = 0, prev_stage = 0, prev_ph = 0, q_key = -1;
             bool ok = true;
-            for (int w = w0; w < w1 && ok; ++w) {
-                const Item it = decode_item(p, w, true);
+            Walk wk;
+            walk_init(wk, p, w0);
+            for (; wk.w < w1 && ok; walk_next(wk, p)) {
+                const Item it = walk_item(wk, p, true);
                 if (!it.run) continue;
                 const UnitInfo &u = it.u;
                 for (int c = 0; c < it.n_chunks && ok; ++c) {
@@ -393,8 +439,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             // same rotation, so in-order issue does not starve anyone.
             bool ok = true;
             int A = 0, qcnt = 0, q_key = -1, st = 0, sph = 0;
-            for (int w = w0; w < w1 && ok; ++w) {
-                const Item it = decode_item(p, w, false);
+            Walk wk;
+            walk_init(wk, p, w0);
+            for (; wk.w < w1 && ok; walk_next(wk, p)) {
+                const Item it = walk_item(wk, p, false);
                 if (!it.run) continue;
                 for (int c = 0; c < it.n_chunks && ok; ++c) {
                     const int nqt = min(p.q_tiles, it.n_qt - c * p.q_tiles);
@@ -443,8 +491,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         const float scale2 = mv.scale * kLog2e;
         int A = 0, mine = 0, q_key = -1, epoch = 0;  // mine = accumulators this group has consumed (barrier phase)
         bool ok = true;
-        for (int w = w0; w < w1 && ok; ++w) {
-            const Item it = decode_item(p, w, false);
+        Walk wk;
+        walk_init(wk, p, w0);
+        for (; wk.w < w1 && ok; walk_next(wk, p)) {
+            const Item it = walk_item(wk, p, false);
             if (!it.run) continue;
             const UnitInfo &u = it.u;
             const int t0 = it.t0, t1 = it.t1, sbq = it.sbq, n_sb = it.n_sb;
