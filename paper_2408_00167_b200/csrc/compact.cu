@@ -2,13 +2,15 @@
 //
 // One CTA copies kRowsPerCta output rows of one unit (layer, selection group, request) for every KV head of the
 // group, K and V, as 16-byte pieces: consecutive threads move consecutive pieces of a row, so both the gathered
-// reads (whole rows) and the writes (contiguous rows) are fully coalesced 128-bit accesses.
+// reads (whole rows) and the writes (contiguous rows) are fully coalesced 128-bit accesses.  A CTA takes 256 rows
+// so that the dependent chain in front of the copies (batch metadata -> kept indices -> source addresses) is paid
+// once per 128 KiB moved, and every thread has eight 16-byte loads in flight before its first store.
 #include "finch_internal.cuh"
 
 namespace finch {
 namespace {
 
-constexpr int kRowsPerCta = 32;
+constexpr int kRowsPerCta = 256;  // = kCompactThreads: one thread fetches one kept index
 constexpr int kCompactThreads = 256;
 
 __global__ void __launch_bounds__(kCompactThreads)
@@ -61,17 +63,21 @@ compact_kernel(ModelView mv, BatchView bv, const int *kept_idx, const int *out_l
         char *dst_base = const_cast<char *>(dst.ptr) + ((int64_t)u.l * dst.stride_layer + (int64_t)kvh * dst.stride_head +
                                                         (int64_t)(u.cache0 + i0) * dst.stride_tok) * e + piece * 16;
         const int64_t ca_step = ca.stride_tok * e, ch_step = ch.stride_tok * e, dst_step = dst.stride_tok * e;
-        uint4 v[kRowsPerCta / kRowsInFlight];
+        constexpr int kBatch = 8;  // rows per thread whose loads are issued before the first store
+#pragma unroll 1
+        for (int k0 = 0; k0 * kRowsInFlight < rows; k0 += kBatch) {
+            uint4 v[kBatch];
 #pragma unroll
-        for (int k = 0; k < kRowsPerCta / kRowsInFlight; ++k) {  // all of this thread's loads first ..
-            const int row = ty + k * kRowsInFlight;
-            const int j = row < rows ? src_idx[row] : -1;
-            if (j >= 0) v[k] = __ldg((const uint4 *)(j < u.c ? ca_base + j * ca_step : ch_base + j * ch_step));
-        }
+            for (int k = 0; k < kBatch; ++k) {  // all of this batch's loads first ..
+                const int row = ty + (k0 + k) * kRowsInFlight;
+                const int j = row < rows ? src_idx[row] : -1;
+                if (j >= 0) v[k] = __ldg((const uint4 *)(j < u.c ? ca_base + j * ca_step : ch_base + j * ch_step));
+            }
 #pragma unroll
-        for (int k = 0; k < kRowsPerCta / kRowsInFlight; ++k) {  // .. then its stores
-            const int row = ty + k * kRowsInFlight;
-            if (row < rows && src_idx[row] >= 0) *(uint4 *)(dst_base + row * dst_step) = v[k];
+            for (int k = 0; k < kBatch; ++k) {  // .. then its stores
+                const int row = ty + (k0 + k) * kRowsInFlight;
+                if (row < rows && src_idx[row] >= 0) *(uint4 *)(dst_base + row * dst_step) = v[k];
+            }
         }
     }
 }
