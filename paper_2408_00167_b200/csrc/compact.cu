@@ -18,6 +18,7 @@ compact_kernel(ModelView mv, BatchView bv, const int *kept_idx, const int *out_l
                TensorView cache_v, const int *cache_pos, TensorView chunk_k, TensorView chunk_v, const int *chunk_pos,
                TensorView out_k, TensorView out_v, int *out_pos, int *status) {
     __shared__ int src_idx[kRowsPerCta];
+    dependency_wait();  // no early launch of the next kernel: this grid runs in many waves and needs every slot
     const UnitInfo u = unit_info(mv, bv, blockIdx.y, blockIdx.z);
     if (!u.ok) {
         if (threadIdx.x == 0) atomicOr(status, FINCH_DEV_BAD_BATCH);
@@ -93,10 +94,9 @@ cudaError_t launch_compact(const Ctx &ctx, const int *kept_idx, const int *out_l
     const int row_blocks = (bv.max_budget + kRowsPerCta - 1) / kRowsPerCta;
     if (units == 0 || bv.batch == 0 || row_blocks == 0) return cudaSuccess;
     dim3 grid(row_blocks, units, bv.batch);
-    compact_kernel<<<grid, kCompactThreads, 0, stream>>>(mv, bv, kept_idx, out_len, cache_k, cache_v, cache_pos, chunk_k,
-                                                         chunk_v, chunk_pos, out_k, out_v, out_pos, ctx.d_status);
     ctx.launches += 1;
-    return cudaGetLastError();
+    return launch_chained(compact_kernel, grid, dim3(kCompactThreads), 0, stream, mv, bv, kept_idx, out_len, cache_k, cache_v,
+                          cache_pos, chunk_k, chunk_v, chunk_pos, out_k, out_v, out_pos, ctx.d_status);
 }
 
 }  // namespace finch

@@ -80,6 +80,33 @@ __device__ __forceinline__ UnitInfo unit_info(const ModelView &mv, const BatchVi
     return u;
 }
 
+// ---- programmatic dependent launch: the kernels of a step form a chain on one stream.  Launched with the
+// programmatic-serialization attribute, a kernel may be scheduled while its predecessor is still running; it then
+// executes everything that does not touch global memory (barrier set-up, tensor-memory allocation), and blocks
+// in dependency_wait() until the predecessor has completed and its writes are visible.  Every kernel of the chain
+// calls dependency_wait() unconditionally, before its first global access and before any early return, so that
+// completion of a kernel always implies completion of everything before it.  Only kernels whose whole grid is
+// resident at once call dependents_may_launch(): CTAs of the next kernel that arrive early and park in their wait
+// would otherwise hold registers and thread slots that later waves of the running kernel need.
+__device__ __forceinline__ void dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... Params, typename... Args>
+cudaError_t launch_chained(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                           Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, Params(args)...);
+}
+
 // ---- launchers implemented in the kernel files; each returns the cudaError_t of its launches ----
 
 // warp-level dot-product scoring (any dtype, any prompt length).  row_stats [L][Hq][total_q] is scratch that holds

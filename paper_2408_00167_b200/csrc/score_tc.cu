@@ -340,9 +340,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
 
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
-    // this CTA's contiguous range of work items
-    const int w0 = p.bounds ? p.bounds[blockIdx.x] : (int)((int64_t)blockIdx.x * p.n_items / gridDim.x);
-    const int w1 = p.bounds ? p.bounds[blockIdx.x + 1] : (int)((int64_t)(blockIdx.x + 1) * p.n_items / gridDim.x);
     const int64_t rows_total = (int64_t)mv.L * mv.Hq * bv.total_q;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -368,6 +365,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // barriers and tensor memory are set up; everything below reads what earlier kernels of the stream wrote
+    dependency_wait();
+    dependents_may_launch();
+    // this CTA's contiguous range of work items
+    const int w0 = p.bounds ? p.bounds[blockIdx.x] : (int)((int64_t)blockIdx.x * p.n_items / gridDim.x);
+    const int w1 = p.bounds ? p.bounds[blockIdx.x + 1] : (int)((int64_t)(blockIdx.x + 1) * p.n_items / gridDim.x);
 
     // Every role walks the same items and keeps the same running counters (key tiles loaded, query loads,
     // accumulators per group), so barrier phases stay in step across items without any extra handshake.
@@ -634,6 +637,8 @@ plan_items_kernel(TcParams p, int *bounds, int n_ctas) {
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    dependency_wait();
+    dependents_may_launch();
     const unsigned long long ipr = (unsigned long long)mv.L * mv.G * p.splits;  // items per request
     if (tid == 0) {
         carry_s = 0;
@@ -695,6 +700,8 @@ __global__ void __launch_bounds__(128)
 merge_stats_kernel(TcParams p) {
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
+    dependency_wait();
+    dependents_may_launch();
     const int h = blockIdx.y % mv.Hq, l = blockIdx.y / mv.Hq;
     const UnitInfo u = unit_info(mv, bv, l * mv.G + h / mv.hpg, blockIdx.z);
     if (!u.ok || u.n_q < p.min_q || u.N == 0) return;
@@ -728,6 +735,7 @@ __global__ void __launch_bounds__(256)
 combine_scores_kernel(TcParams p) {
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
+    dependency_wait();  // many waves of small CTAs: the next kernel's CTAs must not take their slots early
     const UnitInfo u = unit_info(mv, bv, blockIdx.y, blockIdx.z);
     if (!u.ok || u.n_q < p.min_q) return;
     const int j = blockIdx.x * 256 + threadIdx.x;
@@ -813,18 +821,21 @@ cudaError_t launch_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensorMap &c
     dim3 grid(p.n_items < sms ? p.n_items : sms);  // persistent: one CTA per SM walks a contiguous range of items
     if (bv.batch > 1 && (int)grid.x < kPlanBoundsInts) {  // requests of different sizes: ranges of equal work
         int *bounds = (int *)(p.work_prefix + bv.batch + 1);
-        plan_items_kernel<<<1, 1024, 0, stream>>>(p, bounds, (int)grid.x);
+        e = launch_chained(plan_items_kernel, dim3(1), dim3(1024), 0, stream, p, bounds, (int)grid.x);
+        if (e != cudaSuccess) return e;
         p.bounds = bounds;
         ctx.launches += 1;
     }
-    score_tc_kernel<kLse, D><<<grid, kTcThreads, smem, stream>>>(qm, cm, hm, p);
+    e = launch_chained(score_tc_kernel<kLse, D>, grid, dim3(kTcThreads), smem, stream, qm, cm, hm, p);
+    if (e != cudaSuccess) return e;
     dim3 mgrid((bv.max_q + 127) / 128, mv.L * mv.Hq, bv.batch);
-    merge_stats_kernel<<<mgrid, 128, 0, stream>>>(p);
-    score_tc_kernel<kColsum, D><<<grid, kTcThreads, smem, stream>>>(qm, cm, hm, p);
+    e = launch_chained(merge_stats_kernel, mgrid, dim3(128), 0, stream, p);
+    if (e != cudaSuccess) return e;
+    e = launch_chained(score_tc_kernel<kColsum, D>, grid, dim3(kTcThreads), smem, stream, qm, cm, hm, p);
+    if (e != cudaSuccess) return e;
     dim3 cgrid((bv.max_cache + bv.max_chunk + 255) / 256, mv.L * mv.G, bv.batch);
-    combine_scores_kernel<<<cgrid, 256, 0, stream>>>(p);
     ctx.launches += 4;
-    return cudaGetLastError();
+    return launch_chained(combine_scores_kernel, cgrid, dim3(256), 0, stream, p);
 }
 
 }  // namespace

@@ -27,6 +27,8 @@ select_kernel(ModelView mv, BatchView bv, const float *scores, int *kept_idx, in
     __shared__ int warp_tot[2][kSelWarps];
     __shared__ int sel_digit, sel_above;
 
+    dependency_wait();
+    dependents_may_launch();
     const int unit = blockIdx.x;
     const UnitInfo u = unit_info(mv, bv, unit, blockIdx.y);
     const int N = u.N;
@@ -155,9 +157,9 @@ cudaError_t launch_select(const Ctx &ctx, const float *scores, const BatchView &
     cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     dim3 grid(units, bv.batch);
-    select_kernel<<<grid, kSelThreads, smem, stream>>>(mv, bv, scores, kept_idx, out_len, smem_keys, ctx.d_status);
     ctx.launches += 1;
-    return cudaGetLastError();
+    return launch_chained(select_kernel, grid, dim3(kSelThreads), smem, stream, mv, bv, scores, (int *)kept_idx, out_len,
+                          smem_keys, ctx.d_status);
 }
 
 }  // namespace finch
