@@ -365,9 +365,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    // barriers and tensor memory are set up; everything below reads what earlier kernels of the stream wrote
-    dependency_wait();
-    dependents_may_launch();
+    // Barriers and tensor memory are set up; what follows reads what earlier kernels of the stream wrote.  The
+    // second sweep's loads and MMAs read only the step's inputs, which were complete before the first sweep began;
+    // what its immediate predecessors produce (the merged row statistics) is read by the softmax warps alone, so
+    // only they wait, and the tensor pipe already fills the accumulators while the statistics are being merged.
+    if (MODE == kLse || warp >= 2) {
+        dependency_wait();
+        dependents_may_launch();
+    }
     // this CTA's contiguous range of work items
     const int w0 = p.bounds ? p.bounds[blockIdx.x] : (int)((int64_t)blockIdx.x * p.n_items / gridDim.x);
     const int w1 = p.bounds ? p.bounds[blockIdx.x + 1] : (int)((int64_t)(blockIdx.x + 1) * p.n_items / gridDim.x);
@@ -700,8 +705,8 @@ __global__ void __launch_bounds__(128)
 merge_stats_kernel(TcParams p) {
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
+    dependents_may_launch();  // before the wait: the second sweep's CTAs may take over SMs as the first sweep's retire
     dependency_wait();
-    dependents_may_launch();
     const int h = blockIdx.y % mv.Hq, l = blockIdx.y / mv.Hq;
     const UnitInfo u = unit_info(mv, bv, l * mv.G + h / mv.hpg, blockIdx.z);
     if (!u.ok || u.n_q < p.min_q || u.N == 0) return;
