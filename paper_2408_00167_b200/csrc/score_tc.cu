@@ -723,15 +723,18 @@ merge_stats_kernel(TcParams p) {
             if (!(pm.y > 0.f)) continue;  // a group that saw none of this row's accumulators in this split
             // A part's sum can be as large as 2^127 against a reference that far below its largest logit: move
             // the sum's exponent into the reference first, so that neither factor below leaves the fp32 range.
-            const int e = ilogbf(pm.y);
-            const float px = pm.x + (float)e, py = ldexpf(pm.y, -e);
+            const int bits = __float_as_int(pm.y);  // pm.y >= 1: a normal number
+            const int e = ((bits >> 23) & 0xff) - 127;
+            const float px = pm.x + (float)e, py = __int_as_float((bits & 0x007fffff) | 0x3f800000);
             const float nm = fmaxf(M, px);
             Z = Z * ex2(M - nm) + py * ex2(px - nm);
             M = nm;
         }
     }
-    const int k = ilogbf(Z);
-    p.merged[row] = make_float2(-(M + (float)k), ldexpf(1.0f, k) / Z);
+    // Z = 2^k * [1, 2) after the loop (it is a sum of terms in [1, 2) times factors <= 1, the largest of them 1)
+    const int zbits = __float_as_int(Z);
+    const int k = ((zbits >> 23) & 0xff) - 127;
+    p.merged[row] = make_float2(-(M + (float)k), __fdividef(1.0f, __int_as_float((zbits & 0x007fffff) | 0x3f800000)));
     if (p.row_lse) p.row_lse[row] = (M + log2f(Z)) * kLn2;
 }
 
