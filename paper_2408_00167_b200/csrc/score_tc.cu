@@ -738,22 +738,26 @@ merge_stats_kernel(TcParams p) {
     if (p.row_lse) p.row_lse[row] = (M + log2f(Z)) * kLn2;
 }
 
-// scores = the four groups' partial column sums, added in group order.
+// scores = the four groups' partial column sums, added in group order.  A request without prompt rows has no
+// accumulators and no partial sums: its scores are the empty sum, zero.
 __global__ void __launch_bounds__(256)
 combine_scores_kernel(TcParams p) {
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
     dependency_wait();  // many waves of small CTAs: the next kernel's CTAs must not take their slots early
     const UnitInfo u = unit_info(mv, bv, blockIdx.y, blockIdx.z);
-    if (!u.ok || u.n_q < p.min_q) return;
+    if (!u.ok || (u.n_q > 0 && u.n_q < p.min_q)) return;
     const int j = blockIdx.x * 256 + threadIdx.x;
     if (j >= u.N) return;
     const int64_t cand = (int64_t)bv.total_cache + bv.total_chunk;
     const int64_t off = ((int64_t)u.l * mv.G + u.G) * cand + u.cache0 + u.chunk0 + j;
     const int64_t gstride = (int64_t)mv.L * mv.G * cand;
-    float s = p.score_parts[off];
+    float s = 0.f;
+    if (u.n_q > 0) {
+        s = p.score_parts[off];
 #pragma unroll
-    for (int g = 1; g < kGroups; ++g) s += p.score_parts[g * gstride + off];
+        for (int g = 1; g < kGroups; ++g) s += p.score_parts[g * gstride + off];
+    }
     p.scores[off] = s;
 }
 

@@ -120,6 +120,16 @@ def test_empty_and_degenerate_requests():
     assert res["out_len"].tolist() == [16, 10, 0, 0]
 
 
+def test_request_without_prompt_rows_scores_zero_and_keeps_the_first_rows():
+    # the sum over no prompt rows is zero for every key: all candidates tie and the lowest indices are kept
+    cfg = _small("c3", "bf16", 4, 2, 64, [(70, 9999, 40, 16), (0, 9999, 30, 16), (8, 9999, 20, 16)], planted_frac=0.0)
+    st = wl.steady_state(cfg, [0, 1], step=2)
+    summary, res, _ = _run_and_check(cfg, st, 2)
+    lo = int(st["cache_off"][1] + st["chunk_off"][1])
+    assert np.all(res["scores"][:, :, lo:lo + 46] == 0.0)
+    np.testing.assert_array_equal(res["kept_idx"][:, :, 16:32], np.broadcast_to(np.arange(16), (2, 2, 16)))
+
+
 @pytest.mark.parametrize("budget", [0, 1, 63, 104, 105, 500])
 def test_budget_edges(budget):
     cfg = _small("c3", "bf16", 4, 2, 64, [(12, 9999, 65, 40)])
