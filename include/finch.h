@@ -193,7 +193,10 @@ finch_status finch_step(finch_ctx *ctx, const finch_tensor *prompt_q, const finc
  * pinned memory; they are copied into the caller's DEVICE staging tensors stage_* (which must be dense and of the
  * same shapes), the step runs on them and on the device-resident cache, and kept_idx / out_len are copied back to
  * host_kept_idx [n_layers][G][total_cache] / host_out_len [batch].  The compressed cache (out_k, out_v, out_pos)
- * stays on the device for the next step.  Unlike the other calls this one WAITS for the stream before it returns.
+ * stays on the device for the next step.  The chunk's V rows, which only the compaction reads, and the kept
+ * indices on their way back travel on a second stream that the context owns, ordered against `cuda_stream` by
+ * events, so the scoring kernels run while V is still being copied.  Unlike the other calls this one WAITS, for
+ * both streams, before it returns.
  * The workspace must hold finch_workspace_bytes (scores live there).  Errors as for finch_step, plus
  * FINCH_ERR_BAD_LAYOUT when a staging tensor is not dense. */
 finch_status finch_step_host(finch_ctx *ctx, const void *host_prompt_q, const void *host_chunk_k,

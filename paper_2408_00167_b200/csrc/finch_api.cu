@@ -171,6 +171,8 @@ finch_status finch_ctx_create(const finch_config *cfg, finch_ctx **out) {
     ctx->d_status = nullptr;
     ctx->dry = cfg->device < 0;
     ctx->sm_count = 0;
+    ctx->copy_stream = nullptr;
+    ctx->ev_entry = ctx->ev_v_ready = ctx->ev_selected = nullptr;
     ctx->launches = 0;
     if (!ctx->dry) {
         int n_dev = 0;
@@ -187,9 +189,13 @@ finch_status finch_ctx_create(const finch_config *cfg, finch_ctx **out) {
             delete ctx;
             return FINCH_ERR_OOM;
         }
-        if (cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess) {
-            cudaFree(ctx->d_status);
-            delete ctx;
+        if (cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ctx->ev_entry, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ctx->ev_v_ready, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ctx->ev_selected, cudaEventDisableTiming) != cudaSuccess) {
+            (void)cudaGetLastError();
+            finch_ctx_destroy(ctx);
             return FINCH_ERR_CUDA;
         }
     }
@@ -199,6 +205,10 @@ finch_status finch_ctx_create(const finch_config *cfg, finch_ctx **out) {
 
 void finch_ctx_destroy(finch_ctx *ctx) {
     if (!ctx) return;
+    if (ctx->ev_entry) cudaEventDestroy(ctx->ev_entry);
+    if (ctx->ev_v_ready) cudaEventDestroy(ctx->ev_v_ready);
+    if (ctx->ev_selected) cudaEventDestroy(ctx->ev_selected);
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     if (ctx->d_status) cudaFree(ctx->d_status);
     delete ctx;
 }
@@ -312,31 +322,54 @@ finch_status finch_step_host(finch_ctx *ctx, const void *host_prompt_q, const vo
                               stage_chunk_pos, batch, out_k, out_v, out_pos)))
         return s;
     if (!ws) return FINCH_ERR_INVALID_ARG;
+    if (!aligned16(ws)) return FINCH_ERR_BAD_LAYOUT;
     if (ws_bytes < ws_layout(ctx, batch).total) return FINCH_ERR_WORKSPACE_TOO_SMALL;
     if (ctx->dry) return FINCH_ERR_UNSUPPORTED;
-    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    cudaStream_t stream = (cudaStream_t)cuda_stream, side = ctx->copy_stream;
     const size_t e = mv.elem_bytes;
     const size_t q_bytes = (size_t)mv.L * mv.Hq * batch->total_q * mv.d * e;
     const size_t c_bytes = (size_t)mv.L * mv.Hkv * batch->total_chunk * mv.d * e;
-    cudaError_t ce = cudaSuccess;
-    if (q_bytes) ce = cudaMemcpyAsync(stage_q->ptr, host_prompt_q, q_bytes, cudaMemcpyHostToDevice, stream);
-    if (ce == cudaSuccess && c_bytes)
-        ce = cudaMemcpyAsync(stage_chunk_k->ptr, host_chunk_k, c_bytes, cudaMemcpyHostToDevice, stream);
-    if (ce == cudaSuccess && c_bytes)
-        ce = cudaMemcpyAsync(stage_chunk_v->ptr, host_chunk_v, c_bytes, cudaMemcpyHostToDevice, stream);
-    if (ce == cudaSuccess && batch->total_chunk)
-        ce = cudaMemcpyAsync(stage_chunk_pos, host_chunk_pos, (size_t)batch->total_chunk * 4, cudaMemcpyHostToDevice,
-                             stream);
-    if (ce != cudaSuccess) return FINCH_ERR_CUDA;
-    s = finch_step(ctx, stage_q, cache_k, cache_v, cache_pos, stage_chunk_k, stage_chunk_v, stage_chunk_pos, batch, out_k,
-                   out_v, out_pos, kept_idx, out_len, nullptr, ws, ws_bytes, cuda_stream);
-    if (s) return s;
+    const WsLayout w = ws_layout(ctx, batch);
+    float2 *row_stats = (float2 *)((char *)ws + w.lse_off);
+    float *scores = (float *)((char *)ws + w.scores_off);
+    const BatchView bv = view_of(batch);
+    // The scoring kernels read Q and the chunk's K; only the compaction reads the chunk's V.  V therefore travels
+    // on the side stream, behind everything already enqueued on the caller's stream (an earlier step's compaction
+    // may still be reading the staging tensor), and the compaction waits for it.  The kept indices go back to the
+    // host on the side stream too, while the compaction runs.
+    auto ok = [](cudaError_t ce) { return ce == cudaSuccess; };
+    bool good = ok(cudaEventRecord(ctx->ev_entry, stream)) && ok(cudaStreamWaitEvent(side, ctx->ev_entry, 0));
+    if (good && q_bytes) good = ok(cudaMemcpyAsync(stage_q->ptr, host_prompt_q, q_bytes, cudaMemcpyHostToDevice, stream));
+    if (good && c_bytes)
+        good = ok(cudaMemcpyAsync(stage_chunk_k->ptr, host_chunk_k, c_bytes, cudaMemcpyHostToDevice, stream));
+    if (good && batch->total_chunk)
+        good = ok(cudaMemcpyAsync(stage_chunk_pos, host_chunk_pos, (size_t)batch->total_chunk * 4,
+                                  cudaMemcpyHostToDevice, stream));
+    if (good && c_bytes)
+        good = ok(cudaMemcpyAsync(stage_chunk_v->ptr, host_chunk_v, c_bytes, cudaMemcpyHostToDevice, side));
+    good = good && ok(cudaEventRecord(ctx->ev_v_ready, side));
+    if (good)
+        good = ok(run_score(*ctx, view_of(stage_q), view_of(cache_k), view_of(stage_chunk_k), bv, scores, row_stats,
+                            w.lse_bytes / sizeof(float2), nullptr, stream));
+    if (good) good = ok(launch_select(*ctx, scores, bv, kept_idx, out_len, stream));
+    good = good && ok(cudaEventRecord(ctx->ev_selected, stream)) && ok(cudaStreamWaitEvent(side, ctx->ev_selected, 0));
     const size_t kept_bytes = (size_t)mv.L * mv.G * batch->total_cache * 4;
-    if (kept_bytes) ce = cudaMemcpyAsync(host_kept_idx, kept_idx, kept_bytes, cudaMemcpyDeviceToHost, stream);
-    if (ce == cudaSuccess && batch->batch)
-        ce = cudaMemcpyAsync(host_out_len, out_len, (size_t)batch->batch * 4, cudaMemcpyDeviceToHost, stream);
-    if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
-    return cuda_status(ce);
+    if (good && kept_bytes) good = ok(cudaMemcpyAsync(host_kept_idx, kept_idx, kept_bytes, cudaMemcpyDeviceToHost, side));
+    if (good && batch->batch)
+        good = ok(cudaMemcpyAsync(host_out_len, out_len, (size_t)batch->batch * 4, cudaMemcpyDeviceToHost, side));
+    good = good && ok(cudaStreamWaitEvent(stream, ctx->ev_v_ready, 0));
+    if (good)
+        good = ok(launch_compact(*ctx, kept_idx, out_len, view_of(cache_k), view_of(cache_v), cache_pos,
+                                 view_of(stage_chunk_k), view_of(stage_chunk_v), stage_chunk_pos, bv, view_of(out_k),
+                                 view_of(out_v), out_pos, stream));
+    // both streams are drained before returning, also after a failure, so that nothing of this call is still in
+    // flight when the caller reuses its buffers
+    const bool drained = ok(cudaStreamSynchronize(side)) & ok(cudaStreamSynchronize(stream));
+    if (!good || !drained) {
+        (void)cudaGetLastError();
+        return FINCH_ERR_CUDA;
+    }
+    return FINCH_OK;
 }
 
 finch_status finch_launch_count(const finch_ctx *ctx, uint64_t *out) {

@@ -40,6 +40,10 @@ struct Ctx {
     bool dry;       // validation-only context: nothing is ever enqueued
     int sm_count;
     mutable uint64_t launches;  // kernels enqueued through this context
+    // finch_step_host only: a second stream carries the chunk's V rows to the device while the scoring kernels,
+    // which do not read them, already run; events tie it to the caller's stream on both sides
+    cudaStream_t copy_stream;
+    cudaEvent_t ev_entry, ev_v_ready, ev_selected;
 };
 
 inline TensorView view_of(const finch_tensor *t) {
