@@ -68,9 +68,11 @@ def _check_storage(a, dtype):
 
 
 def score(dtype, q, cache_k, chunk_k, *, n_q_heads, n_kv_heads, head_dim, group_mode=0, scale=None,
-          q_off, chunk_off, cache_off, cache_len, apply_norm=False, want_lse=False, threads=1):
+          q_off, chunk_off, cache_off, cache_len, apply_norm=False, want_lse=False, threads=1,
+          prompt_self_lse=None):
     """A^agg for every (layer, group, request): returns scores [L][G][total_cand] fp64
-    (and row_lse [L][Hq][total_q] fp64 when want_lse)."""
+    (and row_lse [L][Hq][total_q] fp64 when want_lse).  prompt_self_lse [L][Hq][total_q] (natural log, -inf = no
+    term) adds the prompt's own keys to every row's softmax denominator."""
     for a in (q, cache_k, chunk_k):
         _check_storage(a, dtype)
     q_off, chunk_off, cache_off, cache_len = map(_i32, (q_off, chunk_off, cache_off, cache_len))
@@ -82,12 +84,15 @@ def score(dtype, q, cache_k, chunk_k, *, n_q_heads, n_kv_heads, head_dim, group_
     lse = np.full((L, n_q_heads, int(q_off[batch])), np.nan, dtype=np.float64) if want_lse else None
     if scale is None:
         scale = 1.0 / np.sqrt(float(head_dim))
+    if prompt_self_lse is not None:
+        prompt_self_lse = np.ascontiguousarray(prompt_self_lse, dtype=np.float64)
+        assert prompt_self_lse.shape == (L, n_q_heads, int(q_off[batch]))
     rc = lib().finch_oracle_score(
         ctypes.c_int(DTYPES[dtype]), _p(q), _p(cache_k), _p(chunk_k),
         ctypes.c_int(L), ctypes.c_int(n_q_heads), ctypes.c_int(n_kv_heads), ctypes.c_int(head_dim),
         ctypes.c_int(group_mode), ctypes.c_double(scale), ctypes.c_int(batch),
         _p(q_off), _p(chunk_off), _p(cache_off), _p(cache_len), ctypes.c_int(int(apply_norm)),
-        _p(scores), _p(lse), ctypes.c_int(threads))
+        _p(prompt_self_lse), _p(scores), _p(lse), ctypes.c_int(threads))
     if rc:
         raise ValueError(f"finch_oracle_score rc={rc}")
     return (scores, lse) if want_lse else scores

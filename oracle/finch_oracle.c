@@ -22,7 +22,11 @@
  *   cache       keep K,V at the selected positions             (paragraph "Managing the Cache")
  *
  * Readings taken where the paper is silent: the softmax runs over the candidate
- * keys only (rows sum to 1); ties go to the lower candidate index; kept rows
+ * keys only (rows sum to 1) unless the caller supplies, per prompt row, the
+ * log-sum-exp of the row's logits against the prompt's own keys -- in the full
+ * forward pass a prompt row also attends to the prompt ("N = m + n^que + c",
+ * Method, bullet "Extract prompt-guided submatrix"), and with that term the
+ * denominator is the full row's; ties go to the lower candidate index; kept rows
  * are written in ascending candidate order (a flag gives the paper's rank order
  * of its worked example instead); a NaN score ranks below every number.
  *
@@ -77,7 +81,7 @@ static void score_unit(int dtype, const void *q, const void *cache_k, const void
                        int Hq, int Hkv, int d, int group_mode, double scale,
                        int64_t total_q, int64_t total_cache, int64_t total_chunk,
                        int l, int G, int64_t q0, int n_q, int64_t cache0, int c, int64_t chunk0, int m,
-                       int apply_norm, double *out_scores, double *row_lse)
+                       int apply_norm, const double *self_lse, double *out_scores, double *row_lse)
 {
     const int N = c + m;
     const int heads_per_kv = Hq / Hkv;
@@ -111,7 +115,15 @@ static void score_unit(int dtype, const void *q, const void *cache_k, const void
             double Z = 0.0;
             for (int j = 0; j < N; ++j)
                 Z += exp(s[j] - mx);
-            const double lse = mx + log(Z);
+            double lse = mx + log(Z);
+            if (self_lse) {
+                /* the row's keys are the candidates and the prompt's own keys: add the prompt's share,
+                 * exp(self), to the denominator */
+                const double extra = self_lse[(((int64_t)l * Hq + h) * total_q + q0 + p)];
+                const double top = extra > lse ? extra : lse;
+                if (extra > -INFINITY)
+                    lse = top + log(exp(lse - top) + exp(extra - top));
+            }
             if (row_lse)
                 row_lse[(size_t)(h - h_begin) * n_q + p] = lse;
             for (int j = 0; j < N; ++j)
@@ -146,7 +158,8 @@ static int n_groups(int Hkv, int group_mode) { return group_mode == 0 ? Hkv : 1;
 int finch_oracle_score(int dtype, const void *q, const void *cache_k, const void *chunk_k,
                        int L, int Hq, int Hkv, int d, int group_mode, double scale,
                        int batch, const int32_t *q_off, const int32_t *chunk_off, const int32_t *cache_off,
-                       const int32_t *cache_len, int apply_norm, double *scores, double *row_lse, int threads)
+                       const int32_t *cache_len, int apply_norm, const double *prompt_self_lse, double *scores,
+                       double *row_lse, int threads)
 {
     if (L < 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || d <= 0 || batch < 0)
         return 1;
@@ -169,7 +182,7 @@ int finch_oracle_score(int dtype, const void *q, const void *cache_k, const void
         if (row_lse && n_q > 0)
             lse_unit = (double *)malloc((size_t)heads_per_group * n_q * sizeof(double));
         score_unit(dtype, q, cache_k, chunk_k, Hq, Hkv, d, group_mode, scale, total_q, total_cache, total_chunk,
-                   l, G, q_off[b], n_q, cache_off[b], c, chunk_off[b], m, apply_norm,
+                   l, G, q_off[b], n_q, cache_off[b], c, chunk_off[b], m, apply_norm, prompt_self_lse,
                    scores + ((int64_t)l * Gn + G) * total_cand + cache_off[b] + chunk_off[b], lse_unit);
         if (lse_unit) {
             if (c + m > 0)
@@ -313,7 +326,7 @@ int finch_oracle_step(int dtype, const void *q, const void *cache_k, const void 
                       double *scores_ws, int threads)
 {
     int rc = finch_oracle_score(dtype, q, cache_k, chunk_k, L, Hq, Hkv, d, group_mode, scale, batch, q_off, chunk_off,
-                                cache_off, cache_len, 0, scores_ws, NULL, threads);
+                                cache_off, cache_len, 0, NULL, scores_ws, NULL, threads);
     if (rc)
         return rc;
     rc = finch_oracle_select(scores_ws, L, n_groups(Hkv, group_mode), batch, chunk_off, cache_off, cache_len, budget, 0,

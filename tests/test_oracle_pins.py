@@ -162,6 +162,54 @@ def test_row_lse_matches_definition():
     np.testing.assert_allclose(lse, np.log(np.exp(logits).sum(-1)), rtol=1e-13)
 
 
+def test_prompt_self_term_equals_full_row_softmax_over_candidates_and_prompt_keys():
+    # In the full forward pass a prompt row attends to the candidates and, causally, to the prompt's own keys
+    # ("N = m + n^que + c", Method).  Restated with numpy on the explicit concatenated key set: the candidate columns
+    # of that softmax, summed over rows and heads, must equal the oracle fed with the prompt keys' log-sum-exp only.
+    rng = np.random.default_rng(21)
+    L, Hq, Hkv, nq, c, m, d = 2, 4, 2, 6, 7, 5, 8
+    q, ck, hk, meta = _dense(rng, L, Hq, Hkv, nq, c, m, d)
+    kp = rng.standard_normal((L, Hkv, nq, d)).astype(np.float32)          # the prompt's own keys
+    scale, g = 1.0 / math.sqrt(d), Hq // Hkv
+    cand = np.concatenate([ck[:, :, :c], hk], axis=2).astype(np.float64)
+    keys = np.repeat(np.concatenate([cand, kp.astype(np.float64)], axis=2), g, axis=1)   # [L][Hq][N + nq][d]
+    s = np.einsum("lhpd,lhjd->lhpj", q.astype(np.float64), keys) * scale
+    causal = np.tril(np.ones((nq, nq), bool))                              # prompt row p sees prompt keys t <= p
+    s[..., c + m:] = np.where(causal, s[..., c + m:], -np.inf)
+    w = np.exp(s - s.max(axis=-1, keepdims=True))
+    w /= w.sum(axis=-1, keepdims=True)
+    want = w[..., :c + m].sum(axis=2).reshape(L, Hkv, g, c + m).sum(axis=2)
+    sp = s[..., c + m:]
+    self_lse = sp.max(axis=-1) + np.log(np.exp(sp - sp.max(axis=-1, keepdims=True)).sum(axis=-1))
+    got, lse = _score("f32", q, ck, hk, meta, Hq, Hkv, d, prompt_self_lse=self_lse, want_lse=True)
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-15)
+    full_lse = s.max(axis=-1) + np.log(np.exp(s - s.max(axis=-1, keepdims=True)).sum(axis=-1))
+    np.testing.assert_allclose(lse, full_lse, rtol=1e-12)
+    # the prompt takes its share: the candidates' total is below the number of rows, by exactly the prompt's mass
+    np.testing.assert_allclose(got.sum(axis=-1), (1.0 - w[..., c + m:].sum(axis=-1)).sum(axis=2).reshape(L, Hkv, g).sum(axis=2),
+                               rtol=1e-12)
+    assert np.all(got.sum(axis=-1) < g * nq)
+
+
+def test_prompt_self_term_of_minus_infinity_changes_nothing_and_a_huge_one_takes_everything():
+    rng = np.random.default_rng(22)
+    q, ck, hk, meta = _dense(rng, 1, 2, 2, 3, 4, 4, 8)
+    base, base_lse = _score("f32", q, ck, hk, meta, 2, 2, 8, want_lse=True)
+    none = np.full((1, 2, 3), -np.inf)
+    same, same_lse = _score("f32", q, ck, hk, meta, 2, 2, 8, prompt_self_lse=none, want_lse=True)
+    np.testing.assert_array_equal(same, base)
+    np.testing.assert_array_equal(same_lse, base_lse)
+    # a term equal to the candidates' own log-sum-exp halves every weight
+    half = _score("f32", q, ck, hk, meta, 2, 2, 8, prompt_self_lse=base_lse)
+    np.testing.assert_allclose(half, base / 2, rtol=1e-13)
+    # one row with an overwhelming term drops out of the sum; the other rows are untouched
+    big = none.copy()
+    big[0, 1, 2] = 1e4
+    got = _score("f32", q, ck, hk, meta, 2, 2, 8, prompt_self_lse=big)
+    np.testing.assert_array_equal(got[0, 0], base[0, 0])
+    assert np.all(got[0, 1] < base[0, 1]) and np.all(got[0, 1] > 0)
+
+
 def test_bf16_widening_is_exact():
     # 1.0 + 2^-7 is representable in bfloat16; the dot product must see exactly that value.
     bits = np.array([[[[0x3F81]]]], dtype=np.uint16)              # q = 1.0078125
