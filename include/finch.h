@@ -109,6 +109,13 @@ typedef struct {
     int32_t total_q, total_chunk, total_cache;    /* host copies of q_off[batch], chunk_off[batch], cache_off[batch] */
     int32_t max_q, max_cache, max_chunk, max_budget; /* host upper bounds over the requests (grid sizing)      */
     int32_t min_q;                                /* host lower bound of the prompt lengths; 0 when unknown    */
+    /* Optional (NULL = absent), device, [n_layers][n_q_heads][total_q] fp32, natural log: for every prompt row the
+     * log-sum-exp of its scaled logits against the keys it attends to besides the candidates -- in the paper's
+     * full forward pass the prompt's own (causally visible) keys, "N = m + n^que + c" (Method, bullet "Extract
+     * prompt-guided submatrix").  When given, exp(value) is added to the row's softmax denominator, so the weights
+     * are those of the full attention row and a row's candidate weights sum to less than 1; -inf adds nothing.
+     * Without it the softmax runs over the candidates only.  row_lse then reports the full denominator's log.  */
+    const float *prompt_self_lse;
 } finch_batch;
 
 /* Create a context for one model shape on one device.  Fails with FINCH_ERR_UNSUPPORTED when the device is not
@@ -127,7 +134,8 @@ finch_status finch_workspace_bytes(const finch_ctx *ctx, const finch_batch *batc
 /* Prompt-guided scoring (Method, bullets "Sum over heads", "Extract prompt-guided submatrix", "Selection of top r
  * position" up to A^agg; Background, the attention equation):
  *     s[h,p,j]  = scale * <q[h,p], k[kv(h),j]>          for the candidates j < N_b
- *     w[h,p,j]  = exp(s[h,p,j] - lse[h,p])               softmax over the candidates only
+ *     w[h,p,j]  = exp(s[h,p,j] - lse[h,p])               softmax over the candidates only, or, with
+ *                                                        batch->prompt_self_lse, over candidates and prompt keys
  *     scores[j] = sum over the group's heads h and the prompt rows p of w[h,p,j]
  * The normalisation bullet's factor count(A != 0)/(m+c) is a constant on this path (prompt rows see every
  * candidate) and is not applied.  row_lse may be NULL; the workspace is always required.  Entries of `scores`

@@ -21,6 +21,7 @@ struct BatchView {
     int total_q, total_chunk, total_cache;
     int max_q, max_cache, max_chunk, max_budget;
     int min_q;
+    const float *self_lse;  // optional extra softmax-denominator term per prompt row (natural log), or null
 };
 
 struct ModelView {
@@ -52,7 +53,7 @@ inline TensorView view_of(const finch_tensor *t) {
 inline BatchView view_of(const finch_batch *b) {
     return BatchView{b->batch,       b->q_off,       b->chunk_off, b->cache_off, b->cache_len, b->budget,    b->total_q,
                      b->total_chunk, b->total_cache, b->max_q,     b->max_cache, b->max_chunk, b->max_budget,
-                     b->min_q};
+                     b->min_q,       b->prompt_self_lse};
 }
 
 constexpr float kLog2e = 1.4426950408889634f;

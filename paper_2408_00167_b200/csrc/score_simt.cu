@@ -142,6 +142,14 @@ lse_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, TensorVie
         const int p = p0 + ty + 16 * i;
         if (tx == 0 && p < u.n_q) {
             const int64_t row = ((int64_t)u.l * mv.Hq + h) * bv.total_q + u.q0 + p;
+            if (bv.self_lse) {  // the keys the row attends to besides the candidates: one more term of the sum
+                const float ex = bv.self_lse[row] * kLog2e;
+                if (ex > -INFINITY) {
+                    const float nmx = fmaxf(mx, ex);
+                    sm = sm * exp2f(mx - nmx) + exp2f(ex - nmx);
+                    mx = nmx;
+                }
+            }
             row_stats[row] = make_float2(mx, 1.0f / sm);
             if (row_lse) row_lse[row] = (mx + log2f(sm)) * kLn2;
         }

@@ -731,6 +731,14 @@ merge_stats_kernel(TcParams p) {
             M = nm;
         }
     }
+    if (bv.self_lse) {  // the keys the row attends to besides the candidates: one more part, with sum 1
+        const float px = bv.self_lse[row] * kLog2e;
+        if (px > -INFINITY) {
+            const float nm = fmaxf(M, px);
+            Z = Z * ex2(M - nm) + ex2(px - nm);
+            M = nm;
+        }
+    }
     // Z = 2^k * [1, 2) after the loop (it is a sum of terms in [1, 2) times factors <= 1, the largest of them 1)
     const int zbits = __float_as_int(Z);
     const int k = ((zbits >> 23) & 0xff) - 127;

@@ -90,6 +90,38 @@ def test_wide_logit_range_on_the_tensor_core_path(scale):
         g.close()
 
 
+@pytest.mark.parametrize("dtype,Hq,Hkv,d,reqs,group_mode", [
+    ("bf16", 8, 2, 128, [(130, 9999, 300, 333), (20, 9999, 40, 250)], 0),   # tensor-core path
+    ("f32", 4, 2, 64, [(70, 999, 130, 65), (3, 999, 20, 10)], 0),            # warp-level path
+    ("bf16", 4, 2, 64, [(40, 9999, 90, 70)], 1),                             # per-layer groups (warp-level path)
+])
+def test_prompt_self_term_in_the_softmax_denominator(dtype, Hq, Hkv, d, reqs, group_mode):
+    # the full attention row of a prompt token also covers the prompt's own keys (Method, "N = m + n^que + c"):
+    # their log-sum-exp per row enters the denominator; rows with -inf behave as without the term
+    cfg = _small("c3", dtype, Hq, Hkv, d, reqs, group_mode=group_mode, planted_frac=0.03)
+    st = wl.steady_state(cfg, [0, 1], step=2)
+    rng = np.random.default_rng(5)
+    total_q = int(st["q_off"][-1])
+    _, base_lse = oracle_scores(cfg, st, group_mode=group_mode, want_lse=True)
+    self_lse = base_lse + rng.normal(0.0, 2.0, size=base_lse.shape)      # comparable to the candidates' own mass
+    self_lse[rng.random(self_lse.shape) < 0.2] = -np.inf
+    self_lse = self_lse.astype(np.float32).astype(np.float64)
+    assert self_lse.shape == (2, Hq, total_q)
+    g = GpuStep(cfg, st, 2, group_mode=group_mode, prompt_self_lse=self_lse)
+    try:
+        g.run_parts()
+        assert g.status() == 0
+        res = g.results()
+        ref, ref_lse = oracle_scores(cfg, st, group_mode=group_mode, want_lse=True, prompt_self_lse=self_lse)
+        plain = oracle_scores(cfg, st, group_mode=group_mode)
+        assert np.abs(ref - plain).max() > 0.05                           # the term matters in this test
+        summary = check_parity(cfg, st, res, ref, group_mode=group_mode)
+        assert summary["max_rel_err"] < 1e-4
+        np.testing.assert_allclose(res["row_lse"], ref_lse, rtol=2e-5, atol=2e-5)
+    finally:
+        g.close()
+
+
 def test_row_lse_output_matches_oracle():
     cfg = _small("c3", "bf16", 4, 2, 64, [(9, 9999, 70, 40), (64, 9999, 30, 90)])
     st = wl.steady_state(cfg, [0, 1], step=2)
