@@ -125,8 +125,9 @@ def select(scores, *, chunk_off, cache_off, cache_len, budget, rank_order=False)
 
 
 def compact(dtype, kept_idx, out_len, cache_k, cache_v, cache_pos, chunk_k, chunk_v, chunk_pos, *,
-            n_kv_heads, head_dim, group_mode=0, chunk_off, cache_off, cache_len):
-    """Gather kept rows: returns (out_k, out_v, out_pos) in the cache's packed layout."""
+            n_kv_heads, head_dim, group_mode=0, chunk_off, cache_off, cache_len, rope_theta=0.0, rope_pairing=0):
+    """Gather kept rows: returns (out_k, out_v, out_pos) in the cache's packed layout.  rope_theta > 0 re-rotates the
+    K rows from their candidate index to their output slot (pairing 0: coordinates (t, t + d/2); 1: (2t, 2t + 1))."""
     for a in (cache_k, cache_v, chunk_k, chunk_v):
         _check_storage(a, dtype)
     chunk_off, cache_off, cache_len = map(_i32, (chunk_off, cache_off, cache_len))
@@ -140,7 +141,8 @@ def compact(dtype, kept_idx, out_len, cache_k, cache_v, cache_pos, chunk_k, chun
         ctypes.c_int(DTYPES[dtype]), _p(kept_idx), _p(out_len), _p(cache_k), _p(cache_v), _p(cache_pos),
         _p(chunk_k), _p(chunk_v), _p(chunk_pos), ctypes.c_int(L), ctypes.c_int(n_kv_heads),
         ctypes.c_int(head_dim), ctypes.c_int(group_mode), ctypes.c_int(batch),
-        _p(chunk_off), _p(cache_off), _p(cache_len), _p(out_k), _p(out_v), _p(out_pos))
+        _p(chunk_off), _p(cache_off), _p(cache_len), ctypes.c_double(rope_theta), ctypes.c_int(rope_pairing),
+        _p(out_k), _p(out_v), _p(out_pos))
     if rc:
         raise ValueError(f"finch_oracle_compact rc={rc}")
     return out_k, out_v, out_pos

@@ -276,14 +276,55 @@ int finch_oracle_select(const double *scores, int L, int Gn, int batch,
 
 /* --------------------------------------------------------------- compaction */
 
-/* out_k/out_v [L][Hkv][total_cache][d] (same dtype as the inputs, bit copies),
- * out_pos [L][G][total_cache]; cache_pos [L][G][total_cache], chunk_pos [total_chunk]. */
+/* Round a double to the storage type (round to nearest, ties to even) and store it at element i. */
+static void narrow_store(void *base, int dtype, int64_t i, double x)
+{
+    if (dtype == 0) {
+        ((float *)base)[i] = (float)x;
+        return;
+    }
+    /* bfloat16: 8 significant bits.  Scale the significand to an integer, round it, scale back; the result is
+     * exactly representable in binary32, whose upper half is then the bfloat16 pattern. */
+    float f = 0.0f;
+    if (x != 0.0 && isfinite(x)) {
+        int e;
+        const double sig = frexp(x, &e);          /* |sig| in [0.5, 1) */
+        f = (float)ldexp(rint(ldexp(sig, 8)), e - 8);
+    } else {
+        f = (float)x;
+    }
+    uint32_t bits;
+    memcpy(&bits, &f, sizeof bits);
+    ((uint16_t *)base)[i] = (uint16_t)(bits >> 16);
+}
+
+/* Rotary position embedding moved by `delta` positions (Managing the Cache: a kept key that moves from position j
+ * to slot i is rotated by the cosine and sine of the position difference).  RoFormer's rotation acts on pairs of
+ * coordinates (x, y) with angle delta * theta^(-2t/d) for pair t:  x' = x cos - y sin,  y' = y cos + x sin.
+ * pairing 0: pair t = coordinates (t, t + d/2), the layout of the Llama implementation the paper uses;
+ * pairing 1: pair t = coordinates (2t, 2t + 1), RoFormer's own. */
+static void rerotate_row(int dtype, const void *src, int64_t src_elem, void *dst, int64_t dst_elem, int d,
+                         double theta, int pairing, int delta)
+{
+    for (int t = 0; t < d / 2; ++t) {
+        const int ix = pairing == 0 ? t : 2 * t, iy = pairing == 0 ? t + d / 2 : 2 * t + 1;
+        const double angle = (double)delta * pow(theta, -2.0 * (double)t / (double)d);
+        const double x = widen(src, dtype, src_elem + ix), y = widen(src, dtype, src_elem + iy);
+        narrow_store(dst, dtype, dst_elem + ix, x * cos(angle) - y * sin(angle));
+        narrow_store(dst, dtype, dst_elem + iy, y * cos(angle) + x * sin(angle));
+    }
+}
+
+/* out_k/out_v [L][Hkv][total_cache][d] (same dtype as the inputs), out_pos [L][G][total_cache];
+ * cache_pos [L][G][total_cache], chunk_pos [total_chunk].  V rows and, with rope_theta == 0, K rows are bit copies.
+ * With rope_theta > 0 the K rows are taken to carry rotary embeddings at their candidate index (the cache's rows at
+ * their slots, the chunk's rows after them) and are re-rotated to the slot they land in: delta = i - kept[i]. */
 int finch_oracle_compact(int dtype, const int32_t *kept_idx, const int32_t *out_len,
                          const void *cache_k, const void *cache_v, const int32_t *cache_pos,
                          const void *chunk_k, const void *chunk_v, const int32_t *chunk_pos,
                          int L, int Hkv, int d, int group_mode, int batch,
                          const int32_t *chunk_off, const int32_t *cache_off, const int32_t *cache_len,
-                         void *out_k, void *out_v, int32_t *out_pos)
+                         double rope_theta, int rope_pairing, void *out_k, void *out_v, int32_t *out_pos)
 {
     const int Gn = n_groups(Hkv, group_mode);
     const int kv_per_group = Hkv / Gn;
@@ -305,7 +346,11 @@ int finch_oracle_compact(int dtype, const int32_t *kept_idx, const int32_t *out_
                         const int64_t src = j < c
                                                 ? (((int64_t)l * Hkv + kvh) * total_cache + cache_off[b] + j) * row
                                                 : (((int64_t)l * Hkv + kvh) * total_chunk + chunk_off[b] + (j - c)) * row;
-                        memcpy((char *)out_k + dst, (const char *)(j < c ? cache_k : chunk_k) + src, (size_t)row);
+                        if (rope_theta > 0.0)
+                            rerotate_row(dtype, j < c ? cache_k : chunk_k, src / elem_bytes(dtype), out_k,
+                                         dst / elem_bytes(dtype), d, rope_theta, rope_pairing, i - j);
+                        else
+                            memcpy((char *)out_k + dst, (const char *)(j < c ? cache_k : chunk_k) + src, (size_t)row);
                         memcpy((char *)out_v + dst, (const char *)(j < c ? cache_v : chunk_v) + src, (size_t)row);
                     }
                 }
@@ -334,5 +379,5 @@ int finch_oracle_step(int dtype, const void *q, const void *cache_k, const void 
     if (rc)
         return rc;
     return finch_oracle_compact(dtype, kept_idx, out_len, cache_k, cache_v, cache_pos, chunk_k, chunk_v, chunk_pos, L,
-                                Hkv, d, group_mode, batch, chunk_off, cache_off, cache_len, out_k, out_v, out_pos);
+                                Hkv, d, group_mode, batch, chunk_off, cache_off, cache_len, 0.0, 0, out_k, out_v, out_pos);
 }

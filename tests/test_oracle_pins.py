@@ -327,6 +327,84 @@ def test_paper_worked_cache_example():
     assert sorted(set(positions) - set(ascending.tolist())) == discarded
 
 
+def _rope_numpy(x, pos, theta, pairing):
+    """RoFormer's rotation restated with complex numbers: pair t is the complex number x_t + i y_t, multiplied by
+    exp(i * pos * theta^(-2t/d)).  x: [..., d] float64."""
+    d = x.shape[-1]
+    if pairing == 0:
+        z = x[..., :d // 2] + 1j * x[..., d // 2:]
+    else:
+        z = x[..., 0::2] + 1j * x[..., 1::2]
+    z = z * np.exp(1j * pos * theta ** (-2.0 * np.arange(d // 2) / d))
+    out = np.empty_like(x)
+    if pairing == 0:
+        out[..., :d // 2], out[..., d // 2:] = z.real, z.imag
+    else:
+        out[..., 0::2], out[..., 1::2] = z.real, z.imag
+    return out
+
+
+@pytest.mark.parametrize("pairing", [0, 1])
+def test_rerotation_moves_keys_to_their_new_slots_and_keeps_relative_logits(pairing):
+    # keys carry rotary embeddings at their candidate index; after compaction a kept key must look exactly like the
+    # same raw key embedded at its new slot, so that a query at any position sees the logit of the NEW distance
+    rng = np.random.default_rng(31)
+    L, Hkv, d, c, m, theta = 1, 2, 16, 6, 4, 10000.0
+    raw = rng.standard_normal((L, Hkv, c + m, d))
+    rotated = np.stack([_rope_numpy(raw[:, :, j], j, theta, pairing) for j in range(c + m)], axis=2).astype(np.float32)
+    ck, hk = np.ascontiguousarray(rotated[:, :, :c]), np.ascontiguousarray(rotated[:, :, c:])
+    cv, hv = rng.standard_normal((L, Hkv, c, d)).astype(np.float32), rng.standard_normal((L, Hkv, m, d)).astype(np.float32)
+    kept = np.full((L, Hkv, c), -1, np.int32)
+    kept[0, 0, :4] = [0, 3, 5, 8]
+    kept[0, 1, :4] = [1, 2, 7, 9]
+    meta = dict(chunk_off=[0, m], cache_off=[0, c], cache_len=[c])
+    args = ("f32", kept, [4], ck, cv, np.zeros((L, Hkv, c), np.int32), hk, hv, np.zeros(m, np.int32))
+    out_k, out_v, _ = oracle.compact(*args, n_kv_heads=Hkv, head_dim=d, rope_theta=theta, rope_pairing=pairing, **meta)
+    plain_k, plain_v, _ = oracle.compact(*args, n_kv_heads=Hkv, head_dim=d, **meta)
+    np.testing.assert_array_equal(out_v, plain_v)                          # values are never rotated
+    q_raw = rng.standard_normal(d)
+    for g in range(Hkv):
+        for slot, j in enumerate(kept[0, g, :4]):
+            want = _rope_numpy(raw[0, g, j], slot, theta, pairing)         # the raw key embedded at its new slot
+            np.testing.assert_allclose(out_k[0, g, slot], want, rtol=0, atol=2e-6)
+            np.testing.assert_allclose(np.linalg.norm(out_k[0, g, slot]), np.linalg.norm(raw[0, g, j]), rtol=1e-6)
+            # rotary logits depend on the distance only: a query at position 20 against the moved key
+            q_rot = _rope_numpy(q_raw, 20, theta, pairing)
+            same_distance = _rope_numpy(q_raw, 0, theta, pairing) @ _rope_numpy(raw[0, g, j], slot - 20, theta, pairing)
+            np.testing.assert_allclose(q_rot @ out_k[0, g, slot].astype(np.float64), same_distance, atol=1e-5)
+    # a key that stays where it is (slot 0 <- candidate 0) is copied bit for bit
+    np.testing.assert_array_equal(out_k[0, 0, 0], ck[0, 0, 0])
+    assert not np.array_equal(out_k[0, 0, 1], plain_k[0, 0, 1])
+
+
+def test_rerotation_shifts_of_the_paper_example_and_bf16_rounding():
+    # Managing the Cache: ranking [3, 5, 0] of cache [0..5] moves 3 by -3, 5 by -4 and 0 by +2 when the kept keys are
+    # placed in rank order; the oracle's rotation by exactly these shifts must undo/redo the embedding
+    txt = dict(line.split(":") for line in (GOLDEN / "cache_example.txt").read_text().splitlines()
+               if line and not line.startswith("#"))
+    ranking = [int(x) for x in txt["ranking"].split()]
+    shifts = [int(x) for x in txt["shifts"].split()]
+    rng = np.random.default_rng(32)
+    d, theta = 8, 100.0
+    raw = rng.standard_normal((1, 1, 6, d))
+    rotated = np.stack([_rope_numpy(raw[:, :, j], j, theta, 0) for j in range(6)], axis=2)
+    ck = wl.to_storage(rotated, "bf16")
+    kept = np.array(ranking, np.int32).reshape(1, 1, 3).copy()
+    kept = np.concatenate([kept, np.full((1, 1, 3), -1, np.int32)], axis=2)
+    empty = np.zeros((1, 1, 0, d), np.uint16)
+    out_k, _, _ = oracle.compact("bf16", kept, [3], ck, ck, np.zeros((1, 1, 6), np.int32), empty, empty,
+                                 np.zeros(0, np.int32), n_kv_heads=1, head_dim=d, chunk_off=[0, 0], cache_off=[0, 6],
+                                 cache_len=[6], rope_theta=theta)
+    stored = wl.from_storage(ck, "bf16").astype(np.float64)
+    for slot, (tok, shift) in enumerate(zip(ranking, shifts)):
+        assert slot - tok == shift
+        exact = _rope_numpy(stored[0, 0, tok], shift, theta, 0)
+        got = wl.from_storage(out_k[0, 0, slot], "bf16").astype(np.float64)
+        # the stored value is the exact rotation rounded to bfloat16: within half a unit in the last place
+        assert np.all(np.abs(got - exact) <= np.abs(exact) * 2.0 ** -8 + 1e-30)
+        np.testing.assert_array_equal(out_k[0, 0, slot], wl.to_storage(exact, "bf16"))
+
+
 def test_batched_select_layout_and_budget_clamp():
     rng = np.random.default_rng(12)
     L, G = 2, 3
