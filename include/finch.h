@@ -95,6 +95,14 @@ typedef struct {
     float scale;         /* logit scale; 0 selects 1/sqrt(head_dim) (Background, the attention equation)      */
     int32_t max_batch, max_prompt, max_candidates; /* upper bounds used for validation                        */
     int32_t device;      /* CUDA device ordinal; negative = validation-only context                           */
+    /* Rotary re-positioning of the kept keys (Method, paragraph "Managing the Cache").  rope_theta = 0: K rows are
+     * copied bit for bit.  rope_theta > 0 (the rotary base, 10000 for Llama 2): K rows are taken to carry rotary
+     * embeddings at their candidate index -- the cache's rows at their slots, the chunk's rows after them -- and
+     * the compaction rotates each kept row by (output slot - candidate index) positions, so that it arrives embedded
+     * at its new slot.  rope_pairing 0 rotates coordinate pairs (t, t + head_dim/2), the layout of the Llama
+     * implementation; 1 rotates pairs (2t, 2t + 1), RoFormer's own.  V rows are never rotated.                     */
+    float rope_theta;
+    int32_t rope_pairing;
 } finch_config;
 
 typedef struct {

@@ -39,7 +39,7 @@ class finch_config(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("dtype", C.c_int32), ("group_mode", C.c_int32), ("scale", C.c_float),
                 ("max_batch", C.c_int32), ("max_prompt", C.c_int32), ("max_candidates", C.c_int32),
-                ("device", C.c_int32)]
+                ("device", C.c_int32), ("rope_theta", C.c_float), ("rope_pairing", C.c_int32)]
 
 
 class finch_tensor(C.Structure):
@@ -155,9 +155,10 @@ def make_batch(q_off: Sequence[int], chunk_off: Sequence[int], cache_off: Sequen
 # ------------------------------------------------------------------ the entry points
 
 def finch_ctx_create(n_layers, n_q_heads, n_kv_heads, head_dim, dtype, group_mode=FINCH_GROUP_PER_KV_HEAD, scale=0.0,
-                     max_batch=1, max_prompt=256, max_candidates=8192, device=0) -> C.c_void_p:
+                     max_batch=1, max_prompt=256, max_candidates=8192, device=0, rope_theta=0.0,
+                     rope_pairing=0) -> C.c_void_p:
     cfg = finch_config(n_layers, n_q_heads, n_kv_heads, head_dim, dtype, group_mode, scale, max_batch, max_prompt,
-                       max_candidates, device)
+                       max_candidates, device, rope_theta, rope_pairing)
     ctx = C.c_void_p()
     _check(load().finch_ctx_create(C.byref(cfg), C.byref(ctx)), "finch_ctx_create")
     return ctx

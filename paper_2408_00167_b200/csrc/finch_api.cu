@@ -4,6 +4,8 @@
 #include <new>
 #include <string.h>
 
+#include <vector>
+
 #include "finch_internal.cuh"
 
 using namespace finch;
@@ -152,6 +154,9 @@ finch_status finch_ctx_create(const finch_config *cfg, finch_ctx **out) {
     if (cfg->max_batch <= 0 || cfg->max_prompt <= 0 || cfg->max_candidates <= 0) return FINCH_ERR_INVALID_ARG;
     if (!(cfg->scale >= 0.f) || isinf(cfg->scale)) return FINCH_ERR_INVALID_ARG;
     if (cfg->head_dim % 32 || cfg->head_dim > 256) return FINCH_ERR_UNSUPPORTED;
+    if (!(cfg->rope_theta >= 0.f) || isinf(cfg->rope_theta) || (cfg->rope_theta > 0.f && cfg->rope_theta < 1.f))
+        return FINCH_ERR_INVALID_ARG;
+    if (cfg->rope_pairing != 0 && cfg->rope_pairing != 1) return FINCH_ERR_INVALID_ARG;
     if ((int64_t)cfg->n_layers * cfg->n_kv_heads > 65535 || cfg->max_batch > 65535) return FINCH_ERR_UNSUPPORTED;
 
     finch_ctx *ctx = new (std::nothrow) finch_ctx();
@@ -168,6 +173,10 @@ finch_status finch_ctx_create(const finch_config *cfg, finch_ctx **out) {
     mv.kvpg = mv.Hkv / mv.G;
     mv.scale = cfg->scale > 0.f ? cfg->scale : 1.0f / sqrtf((float)cfg->head_dim);
     mv.elem_bytes = cfg->dtype == FINCH_F32 ? 4 : 2;
+    mv.rope_theta = cfg->rope_theta;
+    mv.rope_pairing = cfg->rope_pairing;
+    mv.rope_table = nullptr;
+    mv.rope_rows = 0;
     ctx->d_status = nullptr;
     ctx->dry = cfg->device < 0;
     ctx->sm_count = 0;
@@ -198,6 +207,26 @@ finch_status finch_ctx_create(const finch_config *cfg, finch_ctx **out) {
             finch_ctx_destroy(ctx);
             return FINCH_ERR_CUDA;
         }
+        if (cfg->rope_theta > 0.f) {
+            // a kept key moves by fewer positions than there are candidates: one table row per distance
+            const int rows = cfg->max_candidates + 1, half = cfg->head_dim / 2;
+            std::vector<float2> table((size_t)rows * half);
+            for (int t = 0; t < half; ++t) {
+                const double inv_freq = pow((double)cfg->rope_theta, -2.0 * t / cfg->head_dim);
+                for (int n = 0; n < rows; ++n)
+                    table[(size_t)n * half + t] = make_float2((float)cos(n * inv_freq), (float)sin(n * inv_freq));
+            }
+            float2 *dev = nullptr;
+            if (cudaMalloc(&dev, table.size() * sizeof(float2)) != cudaSuccess ||
+                cudaMemcpy(dev, table.data(), table.size() * sizeof(float2), cudaMemcpyHostToDevice) != cudaSuccess) {
+                (void)cudaGetLastError();
+                if (dev) cudaFree(dev);
+                finch_ctx_destroy(ctx);
+                return FINCH_ERR_OOM;
+            }
+            mv.rope_table = dev;
+            mv.rope_rows = rows;
+        }
     }
     *out = ctx;
     return FINCH_OK;
@@ -209,6 +238,7 @@ void finch_ctx_destroy(finch_ctx *ctx) {
     if (ctx->ev_v_ready) cudaEventDestroy(ctx->ev_v_ready);
     if (ctx->ev_selected) cudaEventDestroy(ctx->ev_selected);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+    if (ctx->model.rope_table) cudaFree(const_cast<float2 *>(ctx->model.rope_table));
     if (ctx->d_status) cudaFree(ctx->d_status);
     delete ctx;
 }

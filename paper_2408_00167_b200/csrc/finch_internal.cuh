@@ -32,6 +32,12 @@ struct ModelView {
     int kvpg;        // KV heads per selection group
     float scale;     // logit scale (natural units)
     int elem_bytes;  // 2 (bf16) or 4 (f32)
+    float rope_theta;  // rotary base for re-positioning kept keys, 0 = plain copies
+    int rope_pairing;  // 0: pairs (t, t + d/2), 1: pairs (2t, 2t + 1)
+    // (cos, sin) of n * theta^(-2t/d) for n = 0 .. rope_rows - 1 and t = 0 .. d/2 - 1, [rope_rows][d/2]; device
+    // memory owned by the context, computed in double on the host when the context is created
+    const float2 *rope_table;
+    int rope_rows;
 };
 
 struct Ctx {

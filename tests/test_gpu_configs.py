@@ -293,3 +293,55 @@ def test_step_host_matches_step():
         assert e.value.status == fb.FINCH_ERR_BAD_LAYOUT
     finally:
         g.close()
+
+
+@pytest.mark.parametrize("dtype,d,pairing,group_mode", [("bf16", 128, 0, 0), ("bf16", 64, 1, 1), ("f32", 64, 0, 0),
+                                                        ("f32", 32, 1, 0)])
+def test_compact_repositions_rotary_keys(dtype, d, pairing, group_mode):
+    """Managing the Cache: with a rotary base configured, kept K rows are rotated by (output slot - candidate index)
+    positions; V rows, positions and the plain-copy configuration are untouched.  Compared with the fp64 oracle: the
+    GPU rotates in fp32 (angle reduced in double), so a stored value may differ from the oracle's rounding by one unit
+    in the last place of the storage type on rare near-ties, never by more."""
+    import torch
+    rng = np.random.default_rng(7)
+    L, Hkv, theta = 2, 4, 10000.0
+    G = Hkv if group_mode == 0 else 1
+    caps, lens, ms, budgets = [300, 64], [290, 50], [260, 70], [300, 40]
+    cache_off, chunk_off = wl.offsets(caps), wl.offsets(ms)
+    mk = lambda n: wl.to_storage(rng.standard_normal((L, Hkv, n, d)).astype(np.float32), dtype)
+    ck, cv, hk, hv = mk(cache_off[-1]), mk(cache_off[-1]), mk(chunk_off[-1]), mk(chunk_off[-1])
+    cpos = rng.integers(0, 1000, size=(L, G, cache_off[-1])).astype(np.int32)
+    hpos = rng.integers(1000, 2000, size=chunk_off[-1]).astype(np.int32)
+    scores = rng.random((L, G, cache_off[-1] + chunk_off[-1]))
+    kept, out_len = oracle.select(scores, chunk_off=chunk_off, cache_off=cache_off, cache_len=lens, budget=budgets)
+    kw = dict(n_kv_heads=Hkv, head_dim=d, group_mode=group_mode, chunk_off=chunk_off, cache_off=cache_off, cache_len=lens)
+    want_k, want_v, want_p = oracle.compact(dtype, kept, out_len, ck, cv, cpos, hk, hv, hpos, rope_theta=theta,
+                                            rope_pairing=pairing, **kw)
+    plain_k, _, _ = oracle.compact(dtype, kept, out_len, ck, cv, cpos, hk, hv, hpos, **kw)
+    assert not np.array_equal(want_k, plain_k)
+    batch = fb.make_batch(wl.offsets([1, 1]), chunk_off, cache_off, lens, budgets)
+    ctx = fb.finch_ctx_create(L, Hkv, Hkv, d, fb.FINCH_F32 if dtype == "f32" else fb.FINCH_BF16, group_mode,
+                              max_batch=2, max_prompt=1, max_candidates=1024, rope_theta=theta, rope_pairing=pairing)
+    try:
+        dev = lambda a: to_device(a, dtype)
+        out_k, out_v = dev(np.zeros_like(ck)), dev(np.zeros_like(cv))
+        out_pos = torch.full((L, G, int(cache_off[-1])), -1, dtype=torch.int32, device="cuda")
+        fb.finch_compact(ctx, torch.from_numpy(kept).cuda(), torch.from_numpy(out_len).cuda(), dev(ck), dev(cv),
+                         torch.from_numpy(cpos).cuda(), dev(hk), dev(hv), torch.from_numpy(hpos).cuda(), batch,
+                         out_k, out_v, out_pos)
+        assert fb.finch_device_status(ctx) == 0
+        np.testing.assert_array_equal(to_host(out_v, dtype), want_v)
+        np.testing.assert_array_equal(out_pos.cpu().numpy(), want_p)
+        got_bits, want_bits = to_host(out_k, dtype), want_k
+        got = wl.from_storage(got_bits, dtype).astype(np.float64)
+        want = wl.from_storage(want_bits, dtype).astype(np.float64)
+        # fp32 sine, cosine and rotation: an absolute error of a few 1e-7 of the pair's length (bounded here by the
+        # row's), which moves a stored bfloat16 by at most one unit in the last place, and only on near-ties
+        row_scale = np.sqrt((want ** 2).sum(axis=-1, keepdims=True)) + 1e-30
+        if dtype == "bf16":
+            assert np.all(np.abs(got - want) <= np.abs(want) * 2.0 ** -7 + 2e-6 * row_scale)
+            assert np.mean(got_bits != want_bits) < 2e-3                  # nearly all values identical
+        else:
+            assert np.all(np.abs(got - want) <= 2e-6 * row_scale)
+    finally:
+        fb.finch_ctx_destroy(ctx)
