@@ -235,7 +235,7 @@ compact_kernel(ModelView mv, BatchView bv, const int *kept_idx, const int *out_l
         char *dst_base = const_cast<char *>(dst.ptr) + ((int64_t)u.l * dst.stride_layer + (int64_t)kvh * dst.stride_head +
                                                         (int64_t)(u.cache0 + i0) * dst.stride_tok) * e + piece * 16;
         const int64_t ca_step = ca.stride_tok * e, ch_step = ch.stride_tok * e, dst_step = dst.stride_tok * e;
-        constexpr int kBatch = 4;  // rows per thread whose loads are issued before the first store
+        constexpr int kBatch = 8;  // rows per thread whose loads are issued before the first store
 #pragma unroll 1
         for (int k0 = 0; k0 * kRowsInFlight < rows; k0 += kBatch) {
             uint4 v[kBatch];
