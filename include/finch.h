@@ -147,7 +147,7 @@ finch_status finch_workspace_bytes(const finch_ctx *ctx, const finch_batch *batc
  *     scores[j] = sum over the group's heads h and the prompt rows p of w[h,p,j]
  * The normalisation bullet's factor count(A != 0)/(m+c) is a constant on this path (prompt rows see every
  * candidate) and is not applied.  row_lse may be NULL; the workspace is always required.  Entries of `scores`
- * beyond N_b are left untouched.  bf16 inputs (head_dim 64 or 128, one KV head per group) take the tensor-core path,
+ * beyond N_b are left untouched.  bf16 inputs with head_dim 64 or 128 take the tensor-core path (either group mode),
  * everything else warp-level dot products; accumulation, softmax and the column sums are fp32 in a fixed order, so results
  * are run-to-run identical. */
 finch_status finch_score(finch_ctx *ctx, const finch_tensor *prompt_q, const finch_tensor *cache_k,

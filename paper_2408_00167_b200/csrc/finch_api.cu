@@ -55,9 +55,9 @@ WsLayout ws_layout(const finch_ctx *ctx, const finch_batch *b) {
     WsLayout w{};
     const ModelView &mv = ctx->model;
     w.lse_off = 0;
-    const size_t n_scores = (size_t)mv.L * mv.G * ((size_t)b->total_cache + b->total_chunk);
+    const size_t n_kv_scores = (size_t)mv.L * mv.Hkv * ((size_t)b->total_cache + b->total_chunk);
     w.lse_bytes = align_up((size_t)mv.L * mv.Hq * (size_t)b->total_q * sizeof(float2) * (kScoreMaxSplits * 4 + 1) +
-                           (4 * n_scores + 2) * sizeof(float) +  // row statistics, per-group partial scores,
+                           (4 * n_kv_scores + 2) * sizeof(float) +  // row statistics, partial scores per KV head,
                            ((size_t)b->batch + 1) * 8 + 4096);   // and the item plan of a multi-request batch
     w.scores_off = w.lse_off + w.lse_bytes;
     w.scores_bytes = align_up((size_t)mv.L * mv.G * ((size_t)b->total_cache + b->total_chunk) * sizeof(float));
@@ -112,7 +112,7 @@ finch_status validate_compact(const finch_ctx *ctx, const int32_t *kept_idx, con
 
 namespace finch {
 
-// Tensor cores take every request when the context allows them (bf16, supported head_dim, one KV head per group);
+// Tensor cores take every request when the context allows them (bf16, head_dim 64 or 128, either group mode);
 // warp-level dot products take everything else, and also a batch whose tensors the TMA unit cannot describe.
 cudaError_t run_score(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
                       const BatchView &bv, float *scores, float2 *scratch, size_t scratch_capacity, float *row_lse,

@@ -126,7 +126,7 @@ cudaError_t launch_score_simt(const Ctx &ctx, const TensorView &q, const TensorV
                               const BatchView &bv, float *scores, float2 *row_stats, float *row_lse, int nq_below,
                               cudaStream_t stream);
 
-// tensor-core scoring (bf16, head_dim 64 or 128, one KV head per group) for requests with n_q >= min_q.  The scratch
+// tensor-core scoring (bf16, head_dim 64 or 128, either group mode) for requests with n_q >= min_q.  The scratch
 // holds one float2 per prompt row and key split; up to kScoreMaxSplits splits are used when it is large enough.
 constexpr int kScoreMaxSplits = 8;
 bool score_tc_supported(const Ctx &ctx);

@@ -1,4 +1,4 @@
-// Prompt-guided scoring with plain FMA dot products (fp32 inputs, per-layer groups, head dimensions the tensor-core path does not take).
+// Prompt-guided scoring with plain FMA dot products (fp32 inputs, head dimensions the tensor-core path does not take).
 //
 //   lse_simt     one CTA per (64 prompt rows of one query head, unit): sweeps every candidate key and keeps an
 //                online (max, sum-exp) per row -> row_stats = (max of the base-2 logits, 1 / sum), row_lse

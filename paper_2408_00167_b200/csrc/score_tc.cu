@@ -1,4 +1,4 @@
-// Prompt-guided scoring on the 5th-generation tensor cores (bf16 inputs, head_dim 64 or 128, one KV head per group).
+// Prompt-guided scoring on the 5th-generation tensor cores (bf16 inputs, head_dim 64 or 128).
 //
 // One kernel template, two sweeps over the logits S = Q K^T of a unit (layer, KV head, request).  A CTA owns one
 // split of the unit's 128-key tiles and keeps up to four 128-row tiles of the group's prompt queries resident in
@@ -59,6 +59,10 @@ struct TcParams {
     int n_items;       // work items = splits x units x requests, walked by a persistent grid
     const int *bounds;              // [grid + 1] first item of every CTA (work-weighted), or null: equal item counts
     unsigned long long *work_prefix;  // [batch + 1] accumulators of all items of the requests before b (plan scratch)
+    // `mv` is the scoring view: one scoring unit per KV head.  A selection group that spans several KV heads (one
+    // group per layer) is the sum of its heads' units, taken when the partial sums are combined.
+    int out_groups;         // selection groups per layer
+    int units_per_group;    // KV heads (scoring units) per selection group
 };
 
 struct KeyTile {
@@ -746,27 +750,31 @@ merge_stats_kernel(TcParams p) {
     if (p.row_lse) p.row_lse[row] = (M + log2f(Z)) * kLn2;
 }
 
-// scores = the four groups' partial column sums, added in group order.  A request without prompt rows has no
-// accumulators and no partial sums: its scores are the empty sum, zero.
+// scores = the partial column sums of the selection group's KV heads (one scoring unit each), four per head, added in
+// a fixed order: heads ascending, softmax groups ascending.  A request without prompt rows has no accumulators and
+// no partial sums: its scores are the empty sum, zero.
 __global__ void __launch_bounds__(256)
 combine_scores_kernel(TcParams p) {
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
     dependency_wait();  // many waves of small CTAs: the next kernel's CTAs must not take their slots early
-    const UnitInfo u = unit_info(mv, bv, blockIdx.y, blockIdx.z);
+    const int l = blockIdx.y / p.out_groups, og = blockIdx.y % p.out_groups;
+    const UnitInfo u = unit_info(mv, bv, l * mv.G + og * p.units_per_group, blockIdx.z);
     if (!u.ok || (u.n_q > 0 && u.n_q < p.min_q)) return;
     const int j = blockIdx.x * 256 + threadIdx.x;
     if (j >= u.N) return;
     const int64_t cand = (int64_t)bv.total_cache + bv.total_chunk;
-    const int64_t off = ((int64_t)u.l * mv.G + u.G) * cand + u.cache0 + u.chunk0 + j;
+    const int64_t within = u.cache0 + u.chunk0 + j;
     const int64_t gstride = (int64_t)mv.L * mv.G * cand;
     float s = 0.f;
     if (u.n_q > 0) {
-        s = p.score_parts[off];
+        for (int k = 0; k < p.units_per_group; ++k) {
+            const int64_t off = ((int64_t)l * mv.G + og * p.units_per_group + k) * cand + within;
 #pragma unroll
-        for (int g = 1; g < kGroups; ++g) s += p.score_parts[g * gstride + off];
+            for (int g = 0; g < kGroups; ++g) s += p.score_parts[g * gstride + off];
+        }
     }
-    p.scores[off] = s;
+    p.scores[((int64_t)l * p.out_groups + og) * cand + within] = s;
 }
 
 // ------------------------------------------------------------------------------------------------ host side
@@ -825,7 +833,7 @@ template <int D>
 cudaError_t launch_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensorMap &cm, const CUtensorMap &hm, TcParams p,
                      cudaStream_t stream) {
     constexpr int kTileBytes = (D / 64) * kSlabBytes;
-    const ModelView &mv = ctx.model;
+    const ModelView &mv = p.mv;  // the scoring view
     const BatchView &bv = p.bv;
     const int sub_blocks = mv.hpg * ((bv.max_q + kSub - 1) / kSub);
     p.q_tiles = min(kQTiles, (sub_blocks + 1) / 2);
@@ -853,7 +861,7 @@ cudaError_t launch_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensorMap &c
     if (e != cudaSuccess) return e;
     e = launch_chained(score_tc_kernel<kColsum, D>, grid, dim3(kTcThreads), smem, stream, qm, cm, hm, p);
     if (e != cudaSuccess) return e;
-    dim3 cgrid((bv.max_cache + bv.max_chunk + 255) / 256, mv.L * mv.G, bv.batch);
+    dim3 cgrid((bv.max_cache + bv.max_chunk + 255) / 256, mv.L * p.out_groups, bv.batch);
     ctx.launches += 4;
     return launch_chained(combine_scores_kernel, cgrid, dim3(256), 0, stream, p);
 }
@@ -861,7 +869,7 @@ cudaError_t launch_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensorMap &c
 }  // namespace
 
 bool score_tc_supported(const Ctx &ctx) {
-    return ctx.cfg.dtype == FINCH_BF16 && (ctx.model.d == 64 || ctx.model.d == 128) && ctx.model.kvpg == 1;
+    return ctx.cfg.dtype == FINCH_BF16 && (ctx.model.d == 64 || ctx.model.d == 128);
 }
 
 // `partial` holds partial_capacity float2 entries; the key-split count is limited so that one entry per prompt
@@ -870,7 +878,12 @@ bool score_tc_supported(const Ctx &ctx) {
 cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
                             const BatchView &bv, float *scores, float2 *partial, size_t partial_capacity,
                             float *row_lse, int min_q, cudaStream_t stream) {
-    const ModelView &mv = ctx.model;
+    // Scoring works per KV head whatever the selection groups are: a query head only ever meets its own KV head's
+    // keys.  With one selection group per layer the heads' column sums are added when the parts are combined.
+    ModelView mv = ctx.model;
+    mv.G = mv.Hkv;
+    mv.hpg = mv.g;
+    mv.kvpg = 1;
     if (mv.L * mv.G == 0 || bv.batch == 0 || bv.max_q == 0 || bv.max_cache + bv.max_chunk == 0) return cudaSuccess;
     const size_t rows = (size_t)mv.L * mv.Hq * (size_t)bv.total_q;
     // scratch layout (float2 units): per-split, per-group row statistics | merged row statistics | item plan |
@@ -889,7 +902,8 @@ cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorVie
     const int key_tiles = (bv.max_cache + kRows - 1) / kRows + (bv.max_chunk + kRows - 1) / kRows;
     const int max_splits =
         (int)min((size_t)kScoreMaxSplits, ((partial_capacity - parts_f2 - plan_f2) / rows - 1) / kGroups);
-    TcParams p{mv, bv, partial, nullptr, row_lse, scores, nullptr, ctx.d_status, min_q, 1, 2, 1, 0, nullptr, nullptr};
+    TcParams p{mv, bv, partial, nullptr, row_lse, scores, nullptr, ctx.d_status, min_q, 1, 2, 1, 0, nullptr, nullptr,
+               ctx.model.G, ctx.model.kvpg};
     p.splits = choose_splits(mv.L * mv.G * bv.batch, key_tiles, ctx.sm_count > 0 ? ctx.sm_count : 148, max_splits);
     p.merged = partial + (size_t)p.splits * kGroups * rows;
     p.work_prefix = (unsigned long long *)(p.merged + rows);

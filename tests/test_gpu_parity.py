@@ -93,7 +93,8 @@ def test_wide_logit_range_on_the_tensor_core_path(scale):
 @pytest.mark.parametrize("dtype,Hq,Hkv,d,reqs,group_mode", [
     ("bf16", 8, 2, 128, [(130, 9999, 300, 333), (20, 9999, 40, 250)], 0),   # tensor-core path
     ("f32", 4, 2, 64, [(70, 999, 130, 65), (3, 999, 20, 10)], 0),            # warp-level path
-    ("bf16", 4, 2, 64, [(40, 9999, 90, 70)], 1),                             # per-layer groups (warp-level path)
+    ("f32", 4, 2, 32, [(33, 999, 50, 40)], 1),                               # warp-level path, per-layer groups
+    ("bf16", 4, 2, 64, [(40, 9999, 90, 70)], 1),                             # per-layer groups (tensor-core path, heads summed)
 ])
 def test_prompt_self_term_in_the_softmax_denominator(dtype, Hq, Hkv, d, reqs, group_mode):
     # the full attention row of a prompt token also covers the prompt's own keys (Method, "N = m + n^que + c"):
