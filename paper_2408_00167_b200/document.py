@@ -1,0 +1,110 @@
+"""Whole-document compression: the chunk loop around the step (Finch, Section "Method").
+
+"Document Segmentation" feeds the document chunk by chunk; every step scores the compressed cache plus the new chunk
+against the prompt, keeps `budget` candidates and carries them to the next step ("Selection of top r position",
+"Managing the Cache").  This module only orchestrates: two caches on the device that swap roles each step, the batch
+metadata, and the budget schedule.  Every step is one finch_step call; nothing is computed here, and the loop never
+waits for the device (the lengths a step will produce are known on the host: out_len = min(budget, cache + chunk)).
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+from . import binding as fb
+
+
+def fixed_budgets(n_steps: int, k: int) -> List[int]:
+    """The same target size at every step (the cache fills up to k and stays there)."""
+    return [int(k)] * int(n_steps)
+
+
+def paper_budgets(chunk_lens: Sequence[int], sigma: float, k: int) -> List[int]:
+    """The paper's growing schedule, r_{it+1} = m_{it+1} / sigma + c_it, with the final step's r equal to the target
+    size k ("Selection of top r position").  c_it is the cache length after step it (c_0 = 0); the division is
+    rounded down (the paper does not say)."""
+    budgets, c = [], 0
+    for it, m in enumerate(chunk_lens):
+        r = int(m // sigma) + c if it + 1 < len(chunk_lens) else int(k)
+        budgets.append(r)
+        c = min(r, c + int(m))
+    return budgets
+
+
+class DocumentCompressor:
+    """Device-resident state of one batch of documents being compressed.
+
+    capacity[b] rows of cache per request (at least the largest budget that request will see).  `step` takes the
+    chunk's K, V, positions (device tensors in the library's packed layout) and this step's budgets; afterwards
+    `cache_k / cache_v / cache_pos / cache_len` describe the compressed cache.
+    """
+
+    def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: int,
+                 capacity: Sequence[int], max_prompt: int, max_chunk: int, group_mode: int = fb.FINCH_GROUP_PER_KV_HEAD,
+                 scale: float = 0.0, rope_theta: float = 0.0, rope_pairing: int = 0, device="cuda"):
+        import torch
+        self.torch = torch
+        self.device = device
+        self.L, self.Hq, self.Hkv, self.d = n_layers, n_q_heads, n_kv_heads, head_dim
+        self.G = n_kv_heads if group_mode == fb.FINCH_GROUP_PER_KV_HEAD else 1
+        self.capacity = np.asarray(capacity, dtype=np.int32)
+        self.B = len(self.capacity)
+        self.cache_off = np.concatenate([[0], np.cumsum(self.capacity)]).astype(np.int32)
+        total_cap = int(self.cache_off[-1])
+        tdtype = torch.float32 if dtype == fb.FINCH_F32 else torch.bfloat16
+        self.ctx = fb.finch_ctx_create(n_layers, n_q_heads, n_kv_heads, head_dim, dtype, group_mode, scale,
+                                       max_batch=max(self.B, 1), max_prompt=max(max_prompt, 1),
+                                       max_candidates=max(int(self.capacity.max(initial=0)) + max_chunk, 1),
+                                       device=torch.device(device).index or 0, rope_theta=rope_theta,
+                                       rope_pairing=rope_pairing)
+        mk = lambda: dict(k=torch.zeros((n_layers, n_kv_heads, total_cap, head_dim), dtype=tdtype, device=device),
+                          v=torch.zeros((n_layers, n_kv_heads, total_cap, head_dim), dtype=tdtype, device=device),
+                          pos=torch.full((n_layers, self.G, total_cap), -1, dtype=torch.int32, device=device),
+                          len=torch.zeros(max(self.B, 1), dtype=torch.int32, device=device))
+        self._bufs = [mk(), mk()]
+        self._cur = 0
+        self.kept_idx = torch.full((n_layers, self.G, total_cap), -1, dtype=torch.int32, device=device)
+        self.cache_len = np.zeros(self.B, dtype=np.int32)       # host mirror of the device lengths
+        self._ws = None
+        self.steps = 0
+
+    # the cache the next step will read
+    @property
+    def cache_k(self):
+        return self._bufs[self._cur]["k"]
+
+    @property
+    def cache_v(self):
+        return self._bufs[self._cur]["v"]
+
+    @property
+    def cache_pos(self):
+        return self._bufs[self._cur]["pos"]
+
+    def close(self) -> None:
+        if self.ctx:
+            fb.finch_ctx_destroy(self.ctx)
+            self.ctx = None
+
+    def step(self, q, q_off: Sequence[int], chunk_k, chunk_v, chunk_pos, chunk_off: Sequence[int],
+             budget: Sequence[int], scores=None, prompt_self_lse=None) -> None:
+        """One finch_step: [cache ; chunk] -> the other cache.  Enqueues and returns."""
+        torch = self.torch
+        src, dst = self._bufs[self._cur], self._bufs[self._cur ^ 1]
+        budget = np.minimum(np.asarray(budget, dtype=np.int32), self.capacity)
+        batch = fb.make_batch(q_off, chunk_off, self.cache_off, self.cache_len, budget, self.device,
+                              prompt_self_lse=prompt_self_lse)
+        need = fb.finch_workspace_bytes(self.ctx, batch)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+        fb.finch_step(self.ctx, q, src["k"], src["v"], src["pos"], chunk_k, chunk_v, chunk_pos, batch, dst["k"], dst["v"],
+                      dst["pos"], self.kept_idx, dst["len"], scores, self._ws)
+        chunk_len = np.diff(np.asarray(chunk_off, dtype=np.int32))
+        self.cache_len = np.minimum(budget, self.cache_len + chunk_len).astype(np.int32)
+        self._cur ^= 1
+        self.steps += 1
+        self._last_batch = batch      # keeps the metadata tensors alive until the step has run
+
+    def status(self) -> int:
+        return fb.finch_device_status(self.ctx)
