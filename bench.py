@@ -245,6 +245,7 @@ def run_ours(args, cfg: wl.Config):
     h2d = sum(host[k].numel() * host[k].element_size() for k in ("q", "chunk_k", "chunk_v", "chunk_pos"))
     d2h = kept_host.numel() * 4 + len_host.numel() * 4
     fb.finch_ctx_destroy(ctx)
+    document = document_loop(args, cfg, st, dev) if args.document and world == 1 else None
     sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
     chunk_len = np.diff(st["chunk_off"]).astype(np.int64)
     n_cand = st["cache_len"].astype(np.int64) + chunk_len
@@ -280,7 +281,55 @@ def run_ours(args, cfg: wl.Config):
                       "note": "peak = 16 exp2/clk/SM x SMs x sampled SM clock"},
     }
     line["score_alu"]["frac"] = line["score_alu"]["achieved"] / line["score_alu"]["peak"]
+    if document:
+        line["document_loop"] = document
     return line
+
+
+def document_loop(args, cfg: wl.Config, st: dict, dev: dict):
+    """Secondary figure: the whole chunk loop of the configuration's documents (every full chunk, empty cache at
+    the start), caches resident on the device, budgets by the chosen schedule.  The step-1 chunk's K/V stand in for
+    every chunk's data (their distribution is the same); positions advance with the step."""
+    import torch
+    from paper_2408_00167_b200 import binding as fb
+    from paper_2408_00167_b200 import document as doc
+    reqs = cfg.requests
+    n_steps = min(r.text_len // r.chunk for r in reqs)
+    group_mode = cfg.group_mode if args.group_mode < 0 else args.group_mode
+    if args.document == "paper":
+        per_req = [doc.paper_budgets([r.chunk] * n_steps, sigma=r.text_len / r.budget, k=r.budget) for r in reqs]
+    else:
+        per_req = [doc.fixed_budgets(n_steps, r.budget) for r in reqs]
+    drv = doc.DocumentCompressor(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim,
+                                 fb.FINCH_F32 if cfg.dtype == "f32" else fb.FINCH_BF16, [r.budget for r in reqs],
+                                 max_prompt=max(r.n_q for r in reqs), max_chunk=max(r.chunk for r in reqs),
+                                 group_mode=group_mode)
+    chunk_off = st["chunk_off"]
+    pos = [dev["chunk_pos"] + step * max(r.chunk for r in reqs) for step in range(n_steps)]
+
+    def loop():
+        drv.reset()
+        for step in range(n_steps):
+            drv.step(dev["q"], st["q_off"], dev["chunk_k"], dev["chunk_v"], pos[step], chunk_off,
+                     [per_req[b][step] for b in range(len(reqs))])
+    loop()
+    assert drv.status() == 0
+    reps = 5
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record()
+    for _ in range(reps):
+        loop()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / reps
+    assert drv.status() == 0
+    drv.close()
+    tokens = int(n_steps * np.diff(chunk_off).sum())
+    return {"schedule": args.document, "group_mode": "per_layer" if group_mode == 1 else "per_kv_head", "steps": n_steps,
+            "document_tokens": tokens, "ms": ms, "tokens_per_s": tokens / (ms * 1e-3),
+            "final_cache": [int(r.budget) for r in reqs],
+            "note": "whole chunk loop from an empty cache, device-resident caches; one chunk's data reused per step"}
 
 
 def run_reference(args, cfg: wl.Config):
@@ -313,6 +362,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (small profiling runs)")
+    ap.add_argument("--document", default="", choices=["", "fixed", "paper"],
+                    help="also time the whole chunk loop with this budget schedule (adds a document_loop object)")
+    ap.add_argument("--group-mode", type=int, default=-1, choices=[-1, 0, 1],
+                    help="selection groups of the document loop: 0 per KV head, 1 per layer (-1: the configuration's)")
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.config]
     if args.layers > 0:

@@ -82,6 +82,12 @@ class DocumentCompressor:
     def cache_pos(self):
         return self._bufs[self._cur]["pos"]
 
+    def reset(self) -> None:
+        """Start a new batch of documents in the same buffers (empty caches)."""
+        self.cache_len = np.zeros(self.B, dtype=np.int32)
+        self._cur = 0
+        self.steps = 0
+
     def close(self) -> None:
         if self.ctx:
             fb.finch_ctx_destroy(self.ctx)
