@@ -65,7 +65,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     return false;
 }
 
-// ---------------------------------------------------------------- TMA (tiled, 4-D, no multicast)
+// ---------------------------------------------------------------- TMA (tiled, 4-D, one destination CTA)
 __device__ __forceinline__ void tma_load_4d(void *smem_dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2,
                                             int c3) {
     asm volatile(
