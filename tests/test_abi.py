@@ -51,6 +51,10 @@ def _cfg(**kw):
     (dict(scale=-1.0), fb.FINCH_ERR_INVALID_ARG),
     (dict(scale=float("nan")), fb.FINCH_ERR_INVALID_ARG),
     (dict(max_batch=0), fb.FINCH_ERR_INVALID_ARG),
+    (dict(rope_theta=-1.0), fb.FINCH_ERR_INVALID_ARG),
+    (dict(rope_theta=0.5), fb.FINCH_ERR_INVALID_ARG),
+    (dict(rope_theta=float("inf")), fb.FINCH_ERR_INVALID_ARG),
+    (dict(rope_theta=10000.0, rope_pairing=2), fb.FINCH_ERR_INVALID_ARG),
     (dict(head_dim=48), fb.FINCH_ERR_UNSUPPORTED),
     (dict(head_dim=512), fb.FINCH_ERR_UNSUPPORTED),
 ])
@@ -58,6 +62,11 @@ def test_ctx_create_rejects_bad_configs(lib, bad, status):
     with pytest.raises(fb.FinchError) as e:
         fb.finch_ctx_create(**_cfg(**bad))
     assert e.value.status == status
+
+
+def test_ctx_create_accepts_the_rotary_options_without_a_device(lib):
+    ctx = fb.finch_ctx_create(**_cfg(rope_theta=10000.0, rope_pairing=1))     # validation-only: no table is built
+    fb.finch_ctx_destroy(ctx)
 
 
 def test_ctx_create_null_arguments(lib):
