@@ -5,6 +5,8 @@
 // reads (whole rows) and the writes (contiguous rows) are fully coalesced 128-bit accesses.  A CTA takes 256 rows
 // so that the dependent chain in front of the copies (batch metadata -> kept indices -> source addresses) is paid
 // once per 128 KiB moved, and every thread has eight 16-byte loads in flight before its first store.
+#include <cuda_bf16.h>
+
 #include "finch_internal.cuh"
 
 namespace finch {
@@ -19,9 +21,9 @@ constexpr int kCompactThreads = 256;
 // sign), the rotation itself is fp32, the result is rounded to the storage type.
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-__device__ __forceinline__ uint32_t to_bf16(float f) {  // round to nearest even
-    const uint32_t u = __float_as_uint(f);
-    return (u + 0x7fffu + ((u >> 16) & 1u)) >> 16;
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {  // both rounded to nearest even, one instruction
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *(const uint32_t *)&v;
 }
 __device__ __forceinline__ void rotate_pair(float x, float y, float2 cs, float sign, float &xo, float &yo) {
     const float sn = cs.y * sign;
@@ -54,8 +56,8 @@ __device__ __forceinline__ void rotate_pieces(uint4 &px, uint4 &py, const float2
             float x0, y0, x1, y1;
             rotate_pair(bf16_lo(wx[e]), bf16_lo(wy[e]), t[2 * e], sign, x0, y0);
             rotate_pair(bf16_hi(wx[e]), bf16_hi(wy[e]), t[2 * e + 1], sign, x1, y1);
-            wx[e] = to_bf16(x0) | (to_bf16(x1) << 16);
-            wy[e] = to_bf16(y0) | (to_bf16(y1) << 16);
+            wx[e] = pack_bf16(x0, x1);
+            wy[e] = pack_bf16(y0, y1);
         }
     }
 }
@@ -83,7 +85,7 @@ __device__ __forceinline__ void rotate_interleaved(uint4 &pv, const float2 *cs, 
         for (int e = 0; e < 4; ++e) {
             float xo, yo;
             rotate_pair(bf16_lo(w[e]), bf16_hi(w[e]), t[e], sign, xo, yo);
-            w[e] = to_bf16(xo) | (to_bf16(yo) << 16);
+            w[e] = pack_bf16(xo, yo);
         }
     }
 }
