@@ -753,6 +753,8 @@ merge_stats_kernel(TcParams p) {
 // scores = the partial column sums of the selection group's KV heads (one scoring unit each), four per head, added in
 // a fixed order: heads ascending, softmax groups ascending.  A request without prompt rows has no accumulators and
 // no partial sums: its scores are the empty sum, zero.
+constexpr int kCombinePerThread = 4;
+
 __global__ void __launch_bounds__(256)
 combine_scores_kernel(TcParams p) {
     const ModelView &mv = p.mv;
@@ -761,20 +763,30 @@ combine_scores_kernel(TcParams p) {
     const int l = blockIdx.y / p.out_groups, og = blockIdx.y % p.out_groups;
     const UnitInfo u = unit_info(mv, bv, l * mv.G + og * p.units_per_group, blockIdx.z);
     if (!u.ok || (u.n_q > 0 && u.n_q < p.min_q)) return;
-    const int j = blockIdx.x * 256 + threadIdx.x;
-    if (j >= u.N) return;
     const int64_t cand = (int64_t)bv.total_cache + bv.total_chunk;
-    const int64_t within = u.cache0 + u.chunk0 + j;
     const int64_t gstride = (int64_t)mv.L * mv.G * cand;
-    float s = 0.f;
+    // four keys per thread, 256 apart: every load is coalesced and a thread has up to 16 of them in flight
+    float s[kCombinePerThread];
+    int64_t within[kCombinePerThread];
+#pragma unroll
+    for (int i = 0; i < kCombinePerThread; ++i) {
+        const int j = (blockIdx.x * kCombinePerThread + i) * 256 + threadIdx.x;
+        within[i] = j < u.N ? (int64_t)u.cache0 + u.chunk0 + j : -1;
+        s[i] = 0.f;
+    }
     if (u.n_q > 0) {
         for (int k = 0; k < p.units_per_group; ++k) {
-            const int64_t off = ((int64_t)l * mv.G + og * p.units_per_group + k) * cand + within;
+            const int64_t base = ((int64_t)l * mv.G + og * p.units_per_group + k) * cand;
 #pragma unroll
-            for (int g = 0; g < kGroups; ++g) s += p.score_parts[g * gstride + off];
+            for (int g = 0; g < kGroups; ++g)
+#pragma unroll
+                for (int i = 0; i < kCombinePerThread; ++i)
+                    if (within[i] >= 0) s[i] += p.score_parts[g * gstride + base + within[i]];
         }
     }
-    p.scores[((int64_t)l * p.out_groups + og) * cand + within] = s;
+#pragma unroll
+    for (int i = 0; i < kCombinePerThread; ++i)
+        if (within[i] >= 0) p.scores[((int64_t)l * p.out_groups + og) * cand + within[i]] = s[i];
 }
 
 // ------------------------------------------------------------------------------------------------ host side
@@ -861,7 +873,8 @@ cudaError_t launch_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensorMap &c
     if (e != cudaSuccess) return e;
     e = launch_chained(score_tc_kernel<kColsum, D>, grid, dim3(kTcThreads), smem, stream, qm, cm, hm, p);
     if (e != cudaSuccess) return e;
-    dim3 cgrid((bv.max_cache + bv.max_chunk + 255) / 256, mv.L * p.out_groups, bv.batch);
+    dim3 cgrid((bv.max_cache + bv.max_chunk + 256 * kCombinePerThread - 1) / (256 * kCombinePerThread), mv.L * p.out_groups,
+               bv.batch);
     ctx.launches += 4;
     return launch_chained(combine_scores_kernel, cgrid, dim3(256), 0, stream, p);
 }
