@@ -128,7 +128,11 @@ typedef struct {
 
 /* Create a context for one model shape on one device.  Fails with FINCH_ERR_UNSUPPORTED when the device is not
  * compute capability 10.x or the shape is not covered, FINCH_ERR_INVALID_ARG on inconsistent fields
- * (n_q_heads not a multiple of n_kv_heads, non-positive sizes).  *out is set only on success. */
+ * (n_q_heads not a multiple of n_kv_heads, non-positive sizes, a rotary base below 1).  *out is set only on success.
+ * Device memory the context owns, freed by finch_ctx_destroy: a 4-byte status word, a side stream with three events
+ * (used by finch_step_host), and, with rope_theta > 0, the cosine/sine table of the re-positioning,
+ * (max_candidates + 1) x head_dim/2 pairs of fp32 (2 MiB for 4096 candidates and head_dim 128), computed in double
+ * precision on the host during this call. */
 finch_status finch_ctx_create(const finch_config *cfg, finch_ctx **out);
 
 /* Free the context and its status word.  NULL is ignored.  Work still in flight must be synchronised first. */
