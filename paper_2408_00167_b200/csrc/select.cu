@@ -3,7 +3,7 @@
 // One CTA per unit.  Scores are mapped to order-preserving 32-bit keys; four 8-bit radix passes (most significant
 // digit first) locate the key T of the r-th largest score and how many candidates are strictly above it.  A final
 // ordered sweep keeps every candidate above T plus the lowest-indexed candidates equal to T until r are kept, and
-// writes the kept indices in increasing order (block-wide prefix sums over ballots).
+// writes the kept indices in increasing order (two block-wide prefix sums per 4096 candidates).
 #include "finch_internal.cuh"
 
 namespace finch {
@@ -106,40 +106,63 @@ select_kernel(ModelView mv, BatchView bv, const float *scores, int *kept_idx, in
     const uint32_t T = prefix;
     const int ties_to_keep = remaining;  // >= 1
 
-    // ---- ordered sweep: keep key > T, and the first `ties_to_keep` keys == T
+    // ---- ordered sweep: keep key > T, and the first `ties_to_keep` keys == T.  A thread takes four consecutive
+    // candidates, so two block-wide exclusive scans per 4096 candidates (ties before me, kept before me) place every
+    // kept index; the output is ascending by construction.
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    auto block_scan = [&](int v, int *buf, int &total) -> int {  // exclusive prefix of v over the block, in thread order
+        int incl = v;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += up;
+        }
+        if (lane == 31) buf[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            int t = buf[lane];
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, t, off);
+                if (lane >= off) t += up;
+            }
+            buf[lane] = t;  // inclusive totals of the warps
+        }
+        __syncthreads();
+        total = buf[kSelWarps - 1];
+        return (warp ? buf[warp - 1] : 0) + incl - v;
+    };
+    constexpr int kPerThread = 4;
     int base_eq = 0, base_keep = 0;
-    for (int j0 = 0; j0 < N; j0 += kSelThreads) {
-        const int j = j0 + threadIdx.x;
-        const uint32_t k = j < N ? key_at(j) : 0u;
-        const bool gt = j < N && k > T;
-        const bool eq = j < N && k == T;
-        const uint32_t eq_ballot = __ballot_sync(0xffffffffu, eq);
-        if (lane == 0) warp_tot[0][warp] = __popc(eq_ballot);
-        __syncthreads();
-        int eq_before = base_eq, eq_all = 0;
-        for (int w = 0; w < kSelWarps; ++w) {
-            const int t = warp_tot[0][w];
-            if (w < warp) eq_before += t;
-            eq_all += t;
+    for (int j0 = 0; j0 < N; j0 += kSelThreads * kPerThread) {
+        const int j = j0 + threadIdx.x * kPerThread;
+        uint32_t k[kPerThread];
+#pragma unroll
+        for (int e = 0; e < kPerThread; ++e) k[e] = j + e < N ? key_at(j + e) : 0u;
+        int n_eq = 0;
+#pragma unroll
+        for (int e = 0; e < kPerThread; ++e) n_eq += (j + e < N && k[e] == T) ? 1 : 0;
+        int eq_all;
+        int eq_before = base_eq + block_scan(n_eq, warp_tot[0], eq_all);
+        bool keep[kPerThread];
+        int n_keep = 0;
+#pragma unroll
+        for (int e = 0; e < kPerThread; ++e) {
+            const bool in = j + e < N;
+            const bool eq = in && k[e] == T;
+            keep[e] = in && (k[e] > T || (eq && eq_before < ties_to_keep));
+            eq_before += eq ? 1 : 0;
+            n_keep += keep[e] ? 1 : 0;
         }
-        eq_before += __popc(eq_ballot & ((1u << lane) - 1u));
-        const bool keep = gt || (eq && eq_before < ties_to_keep);
-        const uint32_t keep_ballot = __ballot_sync(0xffffffffu, keep);
-        if (lane == 0) warp_tot[1][warp] = __popc(keep_ballot);
-        __syncthreads();
-        int keep_before = base_keep, keep_all = 0;
-        for (int w = 0; w < kSelWarps; ++w) {
-            const int t = warp_tot[1][w];
-            if (w < warp) keep_before += t;
-            keep_all += t;
-        }
-        keep_before += __popc(keep_ballot & ((1u << lane) - 1u));
-        if (keep) kept[keep_before] = j;
+        int keep_all;
+        int slot = base_keep + block_scan(n_keep, warp_tot[1], keep_all);
+#pragma unroll
+        for (int e = 0; e < kPerThread; ++e)
+            if (keep[e]) kept[slot++] = j + e;
         base_eq += eq_all;
         base_keep += keep_all;
-        // no barrier needed here: warp_tot[0] was last read before the second barrier above, and warp_tot[1] is
-        // rewritten only after the next iteration's first barrier
+        // the next iteration's first scan writes warp_tot[0] after this iteration's last barrier, and warp_tot[1]
+        // after two more: every read above has been made by then
     }
 }
 
