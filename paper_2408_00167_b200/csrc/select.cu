@@ -20,7 +20,8 @@ __device__ __forceinline__ uint32_t order_key(float s) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-__global__ void __launch_bounds__(kSelThreads)
+// two CTAs per SM (32 registers per thread): c3's 256 units then run in one wave
+__global__ void __launch_bounds__(kSelThreads, 2)
 select_kernel(ModelView mv, BatchView bv, const float *scores, int *kept_idx, int *out_len, int smem_keys, int *status) {
     extern __shared__ uint32_t key_cache[];  // the first min(N, smem_keys) keys
     __shared__ int hist[256];
@@ -132,6 +133,28 @@ select_kernel(ModelView mv, BatchView bv, const float *scores, int *kept_idx, in
         total = buf[kSelWarps - 1];
         return (warp ? buf[warp - 1] : 0) + incl - v;
     };
+    if (N <= kSelThreads) {
+        // one candidate per thread at most: ballots and the 32 warp totals are cheaper than two scans
+        const int j = threadIdx.x;
+        const uint32_t k = j < N ? key_at(j) : 0u;
+        const bool gt = j < N && k > T;
+        const bool eq = j < N && k == T;
+        const uint32_t eq_ballot = __ballot_sync(0xffffffffu, eq);
+        if (lane == 0) warp_tot[0][warp] = __popc(eq_ballot);
+        __syncthreads();
+        int eq_before = 0;
+        for (int w = 0; w < warp; ++w) eq_before += warp_tot[0][w];
+        eq_before += __popc(eq_ballot & ((1u << lane) - 1u));
+        const bool keep = gt || (eq && eq_before < ties_to_keep);
+        const uint32_t keep_ballot = __ballot_sync(0xffffffffu, keep);
+        if (lane == 0) warp_tot[1][warp] = __popc(keep_ballot);
+        __syncthreads();
+        int keep_before = 0;
+        for (int w = 0; w < warp; ++w) keep_before += warp_tot[1][w];
+        keep_before += __popc(keep_ballot & ((1u << lane) - 1u));
+        if (keep) kept[keep_before] = j;
+        return;
+    }
     constexpr int kPerThread = 4;
     int base_eq = 0, base_keep = 0;
     for (int j0 = 0; j0 < N; j0 += kSelThreads * kPerThread) {
