@@ -113,6 +113,7 @@ def _select_only(scores_np, chunk_lens, cache_caps, cache_lens, budgets, L, G):
 
 
 @pytest.mark.parametrize("n,r,kind", [(1, 1, "rand"), (33, 7, "ties"), (1000, 999, "rand"), (4096, 2048, "ties"),
+                                      (1024, 512, "ties"), (1025, 500, "ties"), (4097, 4000, "special"),
                                       (5000, 1234, "special"), (50000, 30000, "rand"), (50000, 777, "ties")])
 def test_select_matches_oracle_exactly(n, r, kind):
     rng = np.random.default_rng(n * 7 + r)
