@@ -721,9 +721,17 @@ merge_stats_kernel(TcParams p) {
     const int64_t rows_total = (int64_t)mv.L * mv.Hq * bv.total_q;
     const int64_t row = ((int64_t)l * mv.Hq + h) * bv.total_q + u.q0 + pr;
     float M = -INFINITY, Z = 0.f;
-    for (int s = 0; s * tps < k_tiles; ++s) {
-        for (int g = 0; g < kGroups; ++g) {
-            const float2 pm = p.partial[(s * kGroups + g) * rows_total + row];
+    const int n_parts = ((k_tiles + tps - 1) / tps) * kGroups;  // splits that hold key tiles x softmax groups
+    // all loads first (they are independent), eight at a time, then the merge in part order
+#pragma unroll 1
+    for (int i0 = 0; i0 < n_parts; i0 += 8) {
+        float2 part[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            part[i] = i0 + i < n_parts ? p.partial[(int64_t)(i0 + i) * rows_total + row] : make_float2(0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float2 pm = part[i];
             if (!(pm.y > 0.f)) continue;  // a group that saw none of this row's accumulators in this split
             // A part's sum can be as large as 2^127 against a reference that far below its largest logit: move
             // the sum's exponent into the reference first, so that neither factor below leaves the fp32 range.
