@@ -69,10 +69,12 @@ def _check_storage(a, dtype):
 
 def score(dtype, q, cache_k, chunk_k, *, n_q_heads, n_kv_heads, head_dim, group_mode=0, scale=None,
           q_off, chunk_off, cache_off, cache_len, apply_norm=False, want_lse=False, threads=1,
-          prompt_self_lse=None):
+          prompt_self_lse=None, row_limit=None, row_norm=False):
     """A^agg for every (layer, group, request): returns scores [L][G][total_cand] fp64
     (and row_lse [L][Hq][total_q] fp64 when want_lse).  prompt_self_lse [L][Hq][total_q] (natural log, -inf = no
-    term) adds the prompt's own keys to every row's softmax denominator."""
+    term) adds the prompt's own keys to every row's softmax denominator.  row_limit [total_q] int32: row i attends to
+    its request's first row_limit[i] candidates only (causal rows); row_norm scales a row's weights by the fraction of
+    the candidates it sees."""
     for a in (q, cache_k, chunk_k):
         _check_storage(a, dtype)
     q_off, chunk_off, cache_off, cache_len = map(_i32, (q_off, chunk_off, cache_off, cache_len))
@@ -92,7 +94,8 @@ def score(dtype, q, cache_k, chunk_k, *, n_q_heads, n_kv_heads, head_dim, group_
         ctypes.c_int(L), ctypes.c_int(n_q_heads), ctypes.c_int(n_kv_heads), ctypes.c_int(head_dim),
         ctypes.c_int(group_mode), ctypes.c_double(scale), ctypes.c_int(batch),
         _p(q_off), _p(chunk_off), _p(cache_off), _p(cache_len), ctypes.c_int(int(apply_norm)),
-        _p(prompt_self_lse), _p(scores), _p(lse), ctypes.c_int(threads))
+        _p(prompt_self_lse), _p(None if row_limit is None else _i32(row_limit)), ctypes.c_int(int(row_norm)),
+        _p(scores), _p(lse), ctypes.c_int(threads))
     if rc:
         raise ValueError(f"finch_oracle_score rc={rc}")
     return (scores, lse) if want_lse else scores

@@ -26,7 +26,13 @@
  * log-sum-exp of the row's logits against the prompt's own keys -- in the full
  * forward pass a prompt row also attends to the prompt ("N = m + n^que + c",
  * Method, bullet "Extract prompt-guided submatrix"), and with that term the
- * denominator is the full row's; ties go to the lower candidate index; kept rows
+ * denominator is the full row's; query rows may be given a visibility limit
+ * (row i attends to the first limit[i] candidates only: the causal mask of
+ * rows that are themselves document tokens, Method, the positional-bias
+ * paragraph), and then the normalisation can be taken per row: a row's
+ * weights times the fraction of the candidates it sees, which takes the
+ * "score of 1" of a token that only sees itself down to 1/(m+c);
+ * ties go to the lower candidate index; kept rows
  * are written in ascending candidate order (a flag gives the paper's rank order
  * of its worked example instead); a NaN score ranks below every number.
  *
@@ -81,7 +87,8 @@ static void score_unit(int dtype, const void *q, const void *cache_k, const void
                        int Hq, int Hkv, int d, int group_mode, double scale,
                        int64_t total_q, int64_t total_cache, int64_t total_chunk,
                        int l, int G, int64_t q0, int n_q, int64_t cache0, int c, int64_t chunk0, int m,
-                       int apply_norm, const double *self_lse, double *out_scores, double *row_lse)
+                       int apply_norm, const double *self_lse, const int32_t *row_limit, int row_norm,
+                       double *out_scores, double *row_lse)
 {
     const int N = c + m;
     const int heads_per_kv = Hq / Hkv;
@@ -108,12 +115,24 @@ static void score_unit(int dtype, const void *q, const void *cache_k, const void
                     dot += widen(q, dtype, qrow + t) * widen(kbase, dtype, krow + t);
                 s[j] = scale * dot;
             }
+            /* the candidates this row attends to: all of them, or the first row_limit[p] (causal rows) */
+            int vis = N;
+            if (row_limit) {
+                vis = row_limit[q0 + p];
+                if (vis > N)
+                    vis = N;
+                if (vis <= 0) {
+                    if (row_lse)
+                        row_lse[(size_t)(h - h_begin) * n_q + p] = -INFINITY;
+                    continue; /* a row that sees nothing gives nothing */
+                }
+            }
             double mx = s[0];
-            for (int j = 1; j < N; ++j)
+            for (int j = 1; j < vis; ++j)
                 if (s[j] > mx)
                     mx = s[j];
             double Z = 0.0;
-            for (int j = 0; j < N; ++j)
+            for (int j = 0; j < vis; ++j)
                 Z += exp(s[j] - mx);
             double lse = mx + log(Z);
             if (self_lse) {
@@ -126,8 +145,10 @@ static void score_unit(int dtype, const void *q, const void *cache_k, const void
             }
             if (row_lse)
                 row_lse[(size_t)(h - h_begin) * n_q + p] = lse;
-            for (int j = 0; j < N; ++j)
-                A[(size_t)p * N + j] += exp(s[j] - lse);
+            /* per-row reading of the normalisation: count(row != 0) / (m + c) = vis / N */
+            const double row_factor = row_norm ? (double)vis / (double)N : 1.0;
+            for (int j = 0; j < vis; ++j)
+                A[(size_t)p * N + j] += exp(s[j] - lse) * row_factor;
         }
     }
 
@@ -158,8 +179,8 @@ static int n_groups(int Hkv, int group_mode) { return group_mode == 0 ? Hkv : 1;
 int finch_oracle_score(int dtype, const void *q, const void *cache_k, const void *chunk_k,
                        int L, int Hq, int Hkv, int d, int group_mode, double scale,
                        int batch, const int32_t *q_off, const int32_t *chunk_off, const int32_t *cache_off,
-                       const int32_t *cache_len, int apply_norm, const double *prompt_self_lse, double *scores,
-                       double *row_lse, int threads)
+                       const int32_t *cache_len, int apply_norm, const double *prompt_self_lse,
+                       const int32_t *row_limit, int row_norm, double *scores, double *row_lse, int threads)
 {
     if (L < 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || d <= 0 || batch < 0)
         return 1;
@@ -183,7 +204,7 @@ int finch_oracle_score(int dtype, const void *q, const void *cache_k, const void
             lse_unit = (double *)malloc((size_t)heads_per_group * n_q * sizeof(double));
         score_unit(dtype, q, cache_k, chunk_k, Hq, Hkv, d, group_mode, scale, total_q, total_cache, total_chunk,
                    l, G, q_off[b], n_q, cache_off[b], c, chunk_off[b], m, apply_norm, prompt_self_lse,
-                   scores + ((int64_t)l * Gn + G) * total_cand + cache_off[b] + chunk_off[b], lse_unit);
+                   row_limit, row_norm, scores + ((int64_t)l * Gn + G) * total_cand + cache_off[b] + chunk_off[b], lse_unit);
         if (lse_unit) {
             if (c + m > 0)
                 for (int hh = 0; hh < heads_per_group; ++hh)
@@ -371,7 +392,7 @@ int finch_oracle_step(int dtype, const void *q, const void *cache_k, const void 
                       double *scores_ws, int threads)
 {
     int rc = finch_oracle_score(dtype, q, cache_k, chunk_k, L, Hq, Hkv, d, group_mode, scale, batch, q_off, chunk_off,
-                                cache_off, cache_len, 0, NULL, scores_ws, NULL, threads);
+                                cache_off, cache_len, 0, NULL, NULL, 0, scores_ws, NULL, threads);
     if (rc)
         return rc;
     rc = finch_oracle_select(scores_ws, L, n_groups(Hkv, group_mode), batch, chunk_off, cache_off, cache_len, budget, 0,

@@ -210,6 +210,44 @@ def test_prompt_self_term_of_minus_infinity_changes_nothing_and_a_huge_one_takes
     assert np.all(got[0, 1] < base[0, 1]) and np.all(got[0, 1] > 0)
 
 
+def test_causal_rows_equal_a_masked_numpy_softmax_and_the_first_token_scores_one():
+    # Whole-input conditioning (the paper's ablation): the chunk's own tokens are query rows too, each attending to
+    # the cache and to the chunk up to itself; prompt rows see every candidate.  "For the first token, its attention
+    # score is maximal since it only considers itself, leading to a score of 1" (Method, positional bias).
+    rng = np.random.default_rng(41)
+    L, Hq, Hkv, d, c, m, nq = 1, 4, 2, 8, 3, 5, 2
+    rows = m + nq                                                    # chunk rows, then prompt rows
+    q, ck, hk, meta = _dense(rng, L, Hq, Hkv, rows, c, m, d)
+    limit = np.array([c + i + 1 for i in range(m)] + [c + m] * nq, np.int32)
+    got, lse = _score("f32", q, ck, hk, meta, Hq, Hkv, d, row_limit=limit, want_lse=True)
+    g, scale = Hq // Hkv, 1.0 / math.sqrt(d)
+    keys = np.repeat(np.concatenate([ck[:, :, :c], hk], axis=2).astype(np.float64), g, axis=1)
+    s = np.einsum("lhpd,lhjd->lhpj", q.astype(np.float64), keys) * scale
+    visible = np.arange(c + m)[None, :] < limit[:, None]
+    s = np.where(visible, s, -np.inf)
+    w = np.exp(s - s.max(axis=-1, keepdims=True))
+    w /= w.sum(axis=-1, keepdims=True)
+    want = w.sum(axis=2).reshape(L, Hkv, g, c + m).sum(axis=2)
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-15)
+    # per-row normalisation: every row's weights times the fraction of the candidates it sees
+    normed = _score("f32", q, ck, hk, meta, Hq, Hkv, d, row_limit=limit, row_norm=True)
+    want_n = (w * (limit / (c + m))[None, None, :, None]).sum(axis=2).reshape(L, Hkv, g, c + m).sum(axis=2)
+    np.testing.assert_allclose(normed, want_n, rtol=1e-12, atol=1e-15)
+    # the paper's example: with an empty cache the first document token sees only itself and gives it a score of 1
+    q1, ck1, hk1, meta1 = _dense(rng, 1, 1, 1, 4, 0, 4, d)
+    lim1 = np.array([1, 2, 3, 4], np.int32)
+    only_first_row = _score("f32", q1[:, :, :1], ck1, hk1, dict(meta1, q_off=[0, 1]), 1, 1, d, row_limit=lim1[:1])
+    np.testing.assert_array_equal(only_first_row[0, 0], [1.0, 0.0, 0.0, 0.0])
+    scaled = _score("f32", q1[:, :, :1], ck1, hk1, dict(meta1, q_off=[0, 1]), 1, 1, d, row_limit=lim1[:1], row_norm=True)
+    np.testing.assert_array_equal(scaled[0, 0], [0.25, 0.0, 0.0, 0.0])          # count(row != 0) / (m + c) = 1/4
+    # later tokens lose the head start: unnormalised column sums favour early columns, the normalised ones less so
+    full = _score("f32", q1, ck1, hk1, meta1, 1, 1, d, row_limit=lim1)
+    np.testing.assert_allclose(full.sum(), 4.0, rtol=1e-12)                     # four rows, each summing to 1
+    # limits at or beyond N are no limits
+    same = _score("f32", q, ck, hk, meta, Hq, Hkv, d, row_limit=np.full(rows, 99, np.int32))
+    np.testing.assert_array_equal(same, _score("f32", q, ck, hk, meta, Hq, Hkv, d))
+
+
 def test_bf16_widening_is_exact():
     # 1.0 + 2^-7 is representable in bfloat16; the dot product must see exactly that value.
     bits = np.array([[[[0x3F81]]]], dtype=np.uint16)              # q = 1.0078125
