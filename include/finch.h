@@ -124,6 +124,17 @@ typedef struct {
      * are those of the full attention row and a row's candidate weights sum to less than 1; -inf adds nothing.
      * Without it the softmax runs over the candidates only.  row_lse then reports the full denominator's log.  */
     const float *prompt_self_lse;
+    /* Optional (NULL = absent), device, [total_q] int32: query row i of a request attends to that request's first
+     * row_limit[i] candidates only (values are clamped to [0, N_b]; a row with 0 contributes nothing).  This is the
+     * causal mask of query rows that are themselves document tokens -- the paper's ablation that conditions on the
+     * whole input or on the document only instead of the prompt: pass the chunk's queries (and the prompt's) as
+     * prompt_q, with row_limit = cache_len + position in the chunk + 1 for a chunk row and N_b for a prompt row.
+     * With row_norm != 0 every row's weights are multiplied by the fraction of the candidates it sees, the per-row
+     * reading of the Normalization bullet, count(row != 0) / (m + c): a token that sees only itself then scores
+     * 1/(m + c) instead of the "score of 1" of the positional-bias paragraph.  Batches with row_limit take the
+     * warp-level scoring path.                                                                                  */
+    const int32_t *row_limit;
+    int32_t row_norm;
 } finch_batch;
 
 /* Create a context for one model shape on one device.  Fails with FINCH_ERR_UNSUPPORTED when the device is not

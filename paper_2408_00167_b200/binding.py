@@ -52,7 +52,8 @@ class finch_batch(C.Structure):
                 ("cache_len", C.c_void_p), ("budget", C.c_void_p), ("total_q", C.c_int32),
                 ("total_chunk", C.c_int32), ("total_cache", C.c_int32), ("max_q", C.c_int32),
                 ("max_cache", C.c_int32), ("max_chunk", C.c_int32), ("max_budget", C.c_int32),
-                ("min_q", C.c_int32), ("prompt_self_lse", C.c_void_p)]
+                ("min_q", C.c_int32), ("prompt_self_lse", C.c_void_p), ("row_limit", C.c_void_p),
+                ("row_norm", C.c_int32)]
 
 
 class FinchError(RuntimeError):
@@ -122,7 +123,8 @@ class Batch:
     cache_len: object
     budget: object
     c: finch_batch
-    prompt_self_lse: object = None   # keeps the optional device tensor alive
+    prompt_self_lse: object = None   # keeps the optional device tensors alive
+    row_limit: object = None
 
     @property
     def batch(self) -> int:
@@ -130,9 +132,10 @@ class Batch:
 
 
 def make_batch(q_off: Sequence[int], chunk_off: Sequence[int], cache_off: Sequence[int], cache_len: Sequence[int],
-               budget: Sequence[int], device="cuda", prompt_self_lse=None) -> Batch:
+               budget: Sequence[int], device="cuda", prompt_self_lse=None, row_limit=None, row_norm=False) -> Batch:
     """Copy the offset arrays to the device and fill in the host bounds.  prompt_self_lse: optional device tensor
-    [n_layers][n_q_heads][total_q] fp32 (see finch_batch in the header)."""
+    [n_layers][n_q_heads][total_q] fp32; row_limit: optional device tensor [total_q] int32 (see finch_batch in the
+    header)."""
     import torch
     h = [np.ascontiguousarray(a, dtype=np.int32) for a in (q_off, chunk_off, cache_off, cache_len, budget)]
     B = len(h[3])
@@ -148,8 +151,9 @@ def make_batch(q_off: Sequence[int], chunk_off: Sequence[int], cache_off: Sequen
     cb = finch_batch(B, *[x.data_ptr() for x in d], int(h[0][B]), int(h[1][B]), int(h[2][B]),
                      mx(diff(h[0])), mx(h[3]), mx(diff(h[1])), mx(np.minimum(h[4], n_cand)) if B else 0,
                      int(diff(h[0]).min()) if B else 0,
-                     prompt_self_lse.data_ptr() if prompt_self_lse is not None else None)
-    return Batch(*d, cb, prompt_self_lse)
+                     prompt_self_lse.data_ptr() if prompt_self_lse is not None else None,
+                     row_limit.data_ptr() if row_limit is not None else None, int(bool(row_norm)))
+    return Batch(*d, cb, prompt_self_lse, row_limit)
 
 
 # ------------------------------------------------------------------ the entry points

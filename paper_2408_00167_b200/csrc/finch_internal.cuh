@@ -22,6 +22,8 @@ struct BatchView {
     int max_q, max_cache, max_chunk, max_budget;
     int min_q;
     const float *self_lse;  // optional extra softmax-denominator term per prompt row (natural log), or null
+    const int *row_limit;   // optional visible-candidate count per query row [total_q], or null
+    int row_norm;           // scale a row's weights by the fraction of the candidates it sees
 };
 
 struct ModelView {
@@ -59,7 +61,7 @@ inline TensorView view_of(const finch_tensor *t) {
 inline BatchView view_of(const finch_batch *b) {
     return BatchView{b->batch,       b->q_off,       b->chunk_off, b->cache_off, b->cache_len, b->budget,    b->total_q,
                      b->total_chunk, b->total_cache, b->max_q,     b->max_cache, b->max_chunk, b->max_budget,
-                     b->min_q,       b->prompt_self_lse};
+                     b->min_q,       b->prompt_self_lse, b->row_limit, b->row_norm};
 }
 
 constexpr float kLog2e = 1.4426950408889634f;

@@ -95,10 +95,14 @@ lse_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, TensorVie
     const float scale2 = mv.scale * kLog2e;
 
     float run_max[4], run_sum[4];  // base-2 logits, over this thread's own key columns
+    int vis[4];                    // candidates the thread's rows attend to: all, or the row's limit (causal rows)
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         run_max[i] = -INFINITY;
         run_sum[i] = 0.f;
+        const int p = p0 + ty + 16 * i;
+        vis[i] = u.N;
+        if (bv.row_limit && p < u.n_q) vis[i] = max(0, min(u.N, bv.row_limit[u.q0 + p]));
     }
     for (int j0 = 0; j0 < u.N; j0 += kTile) {
         float acc[4][4] = {};
@@ -114,13 +118,13 @@ lse_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, TensorVie
             float tile_max = -INFINITY;
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-                if (j0 + tx + 16 * j < u.N) tile_max = fmaxf(tile_max, acc[i][j] * scale2);
+                if (j0 + tx + 16 * j < vis[i]) tile_max = fmaxf(tile_max, acc[i][j] * scale2);
             if (tile_max == -INFINITY) continue;
             const float new_max = fmaxf(run_max[i], tile_max);
             float sum = run_sum[i] * exp2f(run_max[i] - new_max);  // exp2(-inf) = 0 on the first tile
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-                if (j0 + tx + 16 * j < u.N) sum += exp2f(fmaf(acc[i][j], scale2, -new_max));
+                if (j0 + tx + 16 * j < vis[i]) sum += exp2f(fmaf(acc[i][j], scale2, -new_max));
             run_max[i] = new_max;
             run_sum[i] = sum;
         }
@@ -150,8 +154,12 @@ lse_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, TensorVie
                     mx = nmx;
                 }
             }
-            row_stats[row] = make_float2(mx, 1.0f / sm);
-            if (row_lse) row_lse[row] = (mx + log2f(sm)) * kLn2;
+            // (max, weight per unit of exp2): 1 / sum, times the fraction of the candidates the row sees when the
+            // per-row normalisation is on; a row that sees nothing weighs nothing
+            float w = sm > 0.f ? 1.0f / sm : 0.f;
+            if (bv.row_norm) w *= (float)vis[i] / (float)u.N;
+            row_stats[row] = make_float2(sm > 0.f ? mx : 0.f, w);
+            if (row_lse) row_lse[row] = sm > 0.f ? (mx + log2f(sm)) * kLn2 : -INFINITY;
         }
     }
 }
@@ -191,8 +199,10 @@ colsum_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, Tensor
                 const int p = p0 + ty + 16 * i;
                 if (p >= u.n_q) continue;
                 const float2 st = stats[p];
+                const int lim = bv.row_limit ? bv.row_limit[u.q0 + p] : u.N;  // keys at or beyond it are masked
 #pragma unroll
-                for (int j = 0; j < 4; ++j) col[j] = fmaf(exp2f(fmaf(acc[i][j], scale2, -st.x)), st.y, col[j]);
+                for (int j = 0; j < 4; ++j)
+                    if (j0 + tx + 16 * j < lim) col[j] = fmaf(exp2f(fmaf(acc[i][j], scale2, -st.x)), st.y, col[j]);
             }
         }
     }

@@ -33,7 +33,7 @@ class GpuStep:
     """Device buffers of one step plus the context; `run` calls finch_step, `run_parts` the three calls."""
 
     def __init__(self, cfg: wl.Config, st: dict, n_layers: int, device="cuda", group_mode=None, scale=0.0,
-                 prompt_self_lse=None):
+                 prompt_self_lse=None, row_limit=None, row_norm=False):
         import torch
         self.cfg, self.st, self.dtype, self.device = cfg, st, cfg.dtype, device
         gm = cfg.group_mode if group_mode is None else group_mode
@@ -43,8 +43,11 @@ class GpuStep:
         self_lse = None
         if prompt_self_lse is not None:
             self_lse = torch.from_numpy(np.ascontiguousarray(prompt_self_lse, dtype=np.float32)).to(device)
+        limit = None
+        if row_limit is not None:
+            limit = torch.from_numpy(np.ascontiguousarray(row_limit, dtype=np.int32)).to(device)
         self.batch = fb.make_batch(st["q_off"], st["chunk_off"], st["cache_off"], st["cache_len"], st["budget"],
-                                   device, prompt_self_lse=self_lse)
+                                   device, prompt_self_lse=self_lse, row_limit=limit, row_norm=row_norm)
         c = self.batch.c
         self.ctx = fb.finch_ctx_create(n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim,
                                        fb.FINCH_F32 if cfg.dtype == "f32" else fb.FINCH_BF16, gm, scale,
@@ -94,13 +97,13 @@ class GpuStep:
 
 
 def oracle_scores(cfg: wl.Config, st: dict, group_mode=None, scale=None, threads=8, want_lse=False,
-                  prompt_self_lse=None):
+                  prompt_self_lse=None, row_limit=None, row_norm=False):
     gm = cfg.group_mode if group_mode is None else group_mode
     return oracle.score(cfg.dtype, st["q"], st["cache_k"], st["chunk_k"], n_q_heads=cfg.n_q_heads,
                         n_kv_heads=cfg.n_kv_heads, head_dim=cfg.head_dim, group_mode=gm, scale=scale,
                         q_off=st["q_off"], chunk_off=st["chunk_off"], cache_off=st["cache_off"],
                         cache_len=st["cache_len"], threads=threads, want_lse=want_lse,
-                        prompt_self_lse=prompt_self_lse)
+                        prompt_self_lse=prompt_self_lse, row_limit=row_limit, row_norm=row_norm)
 
 
 def check_parity(cfg: wl.Config, st: dict, res: dict, ref_scores: np.ndarray, group_mode=None, check_scores=True):

@@ -123,6 +123,41 @@ def test_prompt_self_term_in_the_softmax_denominator(dtype, Hq, Hkv, d, reqs, gr
         g.close()
 
 
+@pytest.mark.parametrize("dtype,Hq,Hkv,d,reqs,group_mode,row_norm", [
+    ("bf16", 8, 2, 128, [(150, 9999, 120, 60), (20, 9999, 15, 30)], 0, False),
+    ("bf16", 4, 2, 64, [(90, 9999, 70, 40)], 1, True),
+    ("f32", 4, 4, 32, [(70, 999, 64, 10), (5, 999, 3, 8)], 0, True),
+])
+def test_causal_query_rows_and_per_row_normalisation(dtype, Hq, Hkv, d, reqs, group_mode, row_norm):
+    # the conditioning ablation: the chunk's own tokens are query rows, each seeing the cache and the chunk up to
+    # itself; the last rows of every request stand for prompt rows and see everything; one row sees nothing at all
+    cfg = _small("c3", dtype, Hq, Hkv, d, reqs, group_mode=group_mode, planted_frac=0.03)
+    st = wl.steady_state(cfg, [0, 1], step=2)
+    limit = np.zeros(int(st["q_off"][-1]), np.int32)
+    for b in range(cfg.batch):
+        n_q = int(st["q_off"][b + 1] - st["q_off"][b])
+        c = int(st["cache_len"][b])
+        N = c + int(st["chunk_off"][b + 1] - st["chunk_off"][b])
+        rows = np.minimum(c + np.arange(n_q) + 1, N)
+        rows[-3:] = N + 7                                   # "prompt" rows; a limit beyond N is no limit
+        limit[st["q_off"][b]:st["q_off"][b + 1]] = rows
+    limit[1] = 0                                            # sees nothing: contributes nothing
+    g = GpuStep(cfg, st, 2, group_mode=group_mode, row_limit=limit, row_norm=row_norm)
+    try:
+        g.run_parts()
+        assert g.status() == 0
+        res = g.results()
+        ref, ref_lse = oracle_scores(cfg, st, group_mode=group_mode, want_lse=True, row_limit=limit, row_norm=row_norm)
+        assert np.abs(ref - oracle_scores(cfg, st, group_mode=group_mode)).max() > 0.05
+        summary = check_parity(cfg, st, res, ref, group_mode=group_mode)
+        assert summary["max_rel_err"] < 1e-4
+        finite = np.isfinite(ref_lse)
+        np.testing.assert_allclose(res["row_lse"][finite], ref_lse[finite], rtol=2e-5, atol=2e-5)
+        assert np.all(np.isneginf(res["row_lse"][np.isneginf(ref_lse)]))
+    finally:
+        g.close()
+
+
 def test_row_lse_output_matches_oracle():
     cfg = _small("c3", "bf16", 4, 2, 64, [(9, 9999, 70, 40), (64, 9999, 30, 90)])
     st = wl.steady_state(cfg, [0, 1], step=2)
