@@ -131,8 +131,8 @@ typedef struct {
      * prompt_q, with row_limit = cache_len + position in the chunk + 1 for a chunk row and N_b for a prompt row.
      * With row_norm != 0 every row's weights are multiplied by the fraction of the candidates it sees, the per-row
      * reading of the Normalization bullet, count(row != 0) / (m + c): a token that sees only itself then scores
-     * 1/(m + c) instead of the "score of 1" of the positional-bias paragraph.  Batches with row_limit take the
-     * warp-level scoring path.                                                                                  */
+     * 1/(m + c) instead of the "score of 1" of the positional-bias paragraph.  Both scoring paths take it (the
+     * tensor-core kernels have a masked instantiation that only such batches use).                              */
     const int32_t *row_limit;
     int32_t row_norm;
 } finch_batch;

@@ -117,7 +117,7 @@ namespace finch {
 cudaError_t run_score(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
                       const BatchView &bv, float *scores, float2 *scratch, size_t scratch_capacity, float *row_lse,
                       cudaStream_t stream) {
-    if (score_tc_supported(ctx) && !bv.row_limit) {  // per-row visibility limits: warp-level path only
+    if (score_tc_supported(ctx)) {
         const cudaError_t e = launch_score_tc(ctx, q, cache_k, chunk_k, bv, scores, scratch, scratch_capacity, row_lse,
                                               /*min_q=*/1, stream);
         if (e != cudaErrorNotSupported) return e;

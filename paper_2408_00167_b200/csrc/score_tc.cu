@@ -38,7 +38,8 @@ constexpr int kMaxStages = 4;    // key-tile ring
 constexpr int kTcThreads = 64 + kGroups * 128;
 constexpr int kSlabBytes = kRows * 128;                 // a 64-element (128-byte) wide slab of a 128-row tile
 constexpr int kStatsBytes = 2 * kQTiles * kRows * 8;  // (-ref, weight) of the resident rows, double-buffered
-constexpr int kAuxBytes = 1024 + kStatsBytes;
+constexpr int kLimitBytes = 2 * kQTiles * kRows * 4;  // visible-candidate count of the resident rows (masked variant)
+constexpr int kAuxBytes = 1024 + kStatsBytes + kLimitBytes;
 constexpr int kSmemLimit = 232448;                      // 227 KiB per CTA
 
 enum { kLse = 0, kColsum = 1 };
@@ -188,8 +189,10 @@ __device__ __forceinline__ void lse_chunk(const uint32_t (&r)[32], int nv, float
 
 // `live` is false on lanes whose row of the query tile holds no prompt row: they take part in the (warp-wide)
 // loads but skip the arithmetic, whose input would be whatever the shared memory held before.
+// lane_valid (masked variant): how many of the tile's columns this lane's row attends to; may be <= 0.
+template <bool MASK>
 __device__ __forceinline__ void lse_accumulate(uint32_t taddr, int valid, float scale2, bool live, float &m_raw,
-                                               float &z) {
+                                               float &z, int lane_valid) {
     // one 32-column chunk at a time: with four softmax warps per scheduler the other warps cover the tensor-memory
     // latency, and a single register buffer keeps the kernel inside its register budget
 #pragma unroll 1
@@ -198,15 +201,23 @@ __device__ __forceinline__ void lse_accumulate(uint32_t taddr, int valid, float 
         __syncwarp();
         tmem_ld_x32_issue(taddr + cc * 32, r);
         tmem_ld_x32_wait(r);
-        if (live) lse_chunk(r, valid - cc * 32, scale2, m_raw, z);
+        if (MASK) {
+            const int nv = min(valid, lane_valid) - cc * 32;
+            if (live && nv > 0) lse_chunk(r, nv, scale2, m_raw, z);
+        } else {
+            if (live) lse_chunk(r, valid - cc * 32, scale2, m_raw, z);
+        }
     }
 }
 
 // kColsum: add to (c0, c1) the weights exp2(s * scale2 - ref_r) * w_r of one accumulator row (a key) over the valid
 // prompt rows of the query tile: v0 rows in its first 64-row half, v1 in its second.  The statistics are staged
 // in pairs of rows, (-ref_a, -ref_b, w_a, w_b), so that one 128-bit load feeds two packed operations.
+// Masked variant: lim2 holds, per pair of rows, how many candidates each row attends to; this thread's key has
+// candidate index j and counts for a row only if j is below that row's number.
+template <bool MASK>
 __device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[32], int nv, float scale2, const float4 *sm4, float &c0,
-                                             float &c1) {
+                                             float &c1, const int2 *lim2, int j) {
     float v[32];
 #pragma unroll
     for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]);
@@ -221,13 +232,19 @@ __device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[32], int nv, fl
         const float4 s4 = sm4[e / 2];  // two prompt rows: (-ref_a, -ref_b, w_a, w_b)
         float x0, x1;
         unpack2(fma2(pack2(v[e], v[e + 1]), s2, pack2(s4.x, s4.y)), x0, x1);
+        if (MASK) {
+            const int2 l2 = lim2[e / 2];
+            x0 = j < l2.x ? x0 : -INFINITY;  // exp2(-inf) = 0: the row does not see this key
+            x1 = j < l2.y ? x1 : -INFINITY;
+        }
         acc = fma2(pack2(ex2(x0), ex2(x1)), pack2(s4.z, s4.w), acc);
     }
     unpack2(acc, c0, c1);
 }
 
+template <bool MASK>
 __device__ __forceinline__ void colsum_accumulate(uint32_t taddr, int v0, int v1, float scale2, const float2 *sm,
-                                                  float &c0, float &c1) {
+                                                  float &c0, float &c1, const int *lim, int j) {
     const float4 *sm4 = (const float4 *)sm;
     // chunks 0 and 1 cover the tile's first 64-row half (always present), chunks 2 and 3 the second half
     const int last = v1 > 0 ? 4 : 2;
@@ -237,7 +254,8 @@ __device__ __forceinline__ void colsum_accumulate(uint32_t taddr, int v0, int v1
         __syncwarp();
         tmem_ld_x32_issue(taddr + cc * 32, r);
         tmem_ld_x32_wait(r);
-        colsum_chunk(r, (cc < 2 ? v0 : v1) - (cc & 1) * 32, scale2, sm4 + cc * 16, c0, c1);
+        colsum_chunk<MASK>(r, (cc < 2 ? v0 : v1) - (cc & 1) * 32, scale2, sm4 + cc * 16, c0, c1,
+                           (const int2 *)lim + cc * 16, j);
     }
 }
 
@@ -320,7 +338,9 @@ __device__ __forceinline__ Item walk_item(Walk &k, const TcParams &p, bool repor
     return it;
 }
 
-template <int MODE, int D>
+// MASK: the batch gives every query row a number of candidates it attends to (causal rows); both sweeps then mask
+// the (row, key) pairs beyond it.  The unmasked instantiation contains none of that code.
+template <int MODE, int D, bool MASK>
 __global__ void __launch_bounds__(kTcThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap cache_map,
                 const __grid_constant__ CUtensorMap chunk_map, TcParams p) {
@@ -341,6 +361,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     uint32_t *tmem_slot = (uint32_t *)(stats_ready + 1);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
     float2 *stats_sm = (float2 *)(aux + 1024);  // [2][q_tiles * 128] row statistics, kColsum only
+    int *lim_sm = (int *)(aux + 1024 + kStatsBytes);  // [2][q_tiles * 128] visible candidates per row, masked kColsum
 
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
@@ -518,12 +539,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                 if (MODE == kLse) {
                     float m_raw[kQTiles], z[kQTiles];
                     uint32_t live_mask = 0;  // bit qb: this thread's row of query tile qb holds a prompt row
+                    int lim[kQTiles];        // masked variant: candidates that row attends to
 #pragma unroll
                     for (int k = 0; k < kQTiles; ++k) {
                         m_raw[k] = -INFINITY;
                         z[k] = 0.f;
-                        if (k < nqt && my_row % kSub < sub_block(2 * (qt0 + k) + my_row / kSub, sbq, n_sb, u.n_q).valid)
+                        lim[k] = 0;
+                        const SubBlock sb = sub_block(2 * (qt0 + k) + my_row / kSub, sbq, n_sb, u.n_q);
+                        if (k < nqt && my_row % kSub < sb.valid) {
                             live_mask |= 1u << k;
+                            if (MASK) lim[k] = max(0, min(u.N, bv.row_limit[u.q0 + sb.p0 + my_row % kSub]));
+                        }
                     }
                     for (int t = t0; t < t1 && ok; ++t) {
                         const KeyTile kt = key_tile(u, t);
@@ -535,13 +561,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                             ++mine;
                             tc_fence_after();
                             float mc = 0.f, zc = 0.f;  // the running statistics of query tile qb (kept in registers)
+                            int limc = 0;
 #pragma unroll
                             for (int k = 0; k < kQTiles; ++k)
                                 if (k == qb) {
                                     mc = m_raw[k];
                                     zc = z[k];
+                                    if (MASK) limc = lim[k];
                                 }
-                            lse_accumulate(t_acc, kt.valid, scale2, (live_mask >> qb) & 1u, mc, zc);
+                            lse_accumulate<MASK>(t_acc, kt.valid, scale2, (live_mask >> qb) & 1u, mc, zc, limc - kt.j0);
 #pragma unroll
                             for (int k = 0; k < kQTiles; ++k)
                                 if (k == qb) {
@@ -584,6 +612,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                             float *smf = (float *)dst + (idx >> 1) * 4 + (idx & 1);
                             smf[0] = out.x;
                             smf[2] = out.y;
+                            if (MASK)
+                                lim_sm[(epoch & 1) * kQTiles * kRows + idx] =
+                                    r % kSub < sb.valid ? max(0, min(u.N, bv.row_limit[u.q0 + sb.p0 + r % kSub])) : 0;
                         }
                         __syncwarp();
                         if (lane == 0) mbar_arrive(stats_ready);
@@ -605,7 +636,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                             tc_fence_after();
                             const int v0 = sub_block(2 * (qt0 + qb), sbq, n_sb, u.n_q).valid;
                             const int v1 = sub_block(2 * (qt0 + qb) + 1, sbq, n_sb, u.n_q).valid;
-                            colsum_accumulate(t_acc, v0, v1, scale2, sm + qb * kRows, c0, c1);
+                            colsum_accumulate<MASK>(t_acc, v0, v1, scale2, sm + qb * kRows, c0, c1,
+                                                    lim_sm + ((epoch - 1) & 1) * kQTiles * kRows + qb * kRows,
+                                                    kt.j0 + my_row);
                             tc_fence_before();
                             __syncwarp();
                             if (lane == 0) mbar_arrive(&acc_empty[g]);
@@ -751,10 +784,18 @@ merge_stats_kernel(TcParams p) {
             M = nm;
         }
     }
+    if (!(Z > 0.f)) {  // a row that attends to nothing (its limit is 0) weighs nothing
+        p.merged[row] = make_float2(0.f, 0.f);
+        if (p.row_lse) p.row_lse[row] = -INFINITY;
+        return;
+    }
     // Z = 2^k * [1, 2) after the loop (it is a sum of terms in [1, 2) times factors <= 1, the largest of them 1)
     const int zbits = __float_as_int(Z);
     const int k = ((zbits >> 23) & 0xff) - 127;
-    p.merged[row] = make_float2(-(M + (float)k), __fdividef(1.0f, __int_as_float((zbits & 0x007fffff) | 0x3f800000)));
+    float w = __fdividef(1.0f, __int_as_float((zbits & 0x007fffff) | 0x3f800000));
+    if (bv.row_limit && bv.row_norm)  // per-row normalisation: times the fraction of the candidates the row sees
+        w *= (float)max(0, min(u.N, bv.row_limit[u.q0 + pr])) / (float)u.N;
+    p.merged[row] = make_float2(-(M + (float)k), w);
     if (p.row_lse) p.row_lse[row] = (M + log2f(Z)) * kLn2;
 }
 
@@ -849,7 +890,7 @@ int choose_splits(int ctas_per_split, int key_tiles, int sm_count, int max_split
     return best;
 }
 
-template <int D>
+template <int D, bool MASK>
 cudaError_t launch_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensorMap &cm, const CUtensorMap &hm, TcParams p,
                      cudaStream_t stream) {
     constexpr int kTileBytes = (D / 64) * kSlabBytes;
@@ -860,9 +901,9 @@ cudaError_t launch_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensorMap &c
     p.stages = min(kMaxStages, (kSmemLimit - 1024 - kAuxBytes - p.q_tiles * kTileBytes) / kTileBytes);
     if (p.stages < 2) return cudaErrorNotSupported;
     const int smem = 1024 + (p.q_tiles + p.stages) * kTileBytes + kAuxBytes;
-    cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<kLse, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<kLse, D, MASK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(score_tc_kernel<kColsum, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    e = cudaFuncSetAttribute(score_tc_kernel<kColsum, D, MASK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     p.n_items = p.splits * mv.L * mv.G * bv.batch;
     const int sms = ctx.sm_count > 0 ? ctx.sm_count : 148;
@@ -874,12 +915,12 @@ cudaError_t launch_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensorMap &c
         p.bounds = bounds;
         ctx.launches += 1;
     }
-    e = launch_chained(score_tc_kernel<kLse, D>, grid, dim3(kTcThreads), smem, stream, qm, cm, hm, p);
+    e = launch_chained(score_tc_kernel<kLse, D, MASK>, grid, dim3(kTcThreads), smem, stream, qm, cm, hm, p);
     if (e != cudaSuccess) return e;
     dim3 mgrid((bv.max_q + 127) / 128, mv.L * mv.Hq, bv.batch);
     e = launch_chained(merge_stats_kernel, mgrid, dim3(128), 0, stream, p);
     if (e != cudaSuccess) return e;
-    e = launch_chained(score_tc_kernel<kColsum, D>, grid, dim3(kTcThreads), smem, stream, qm, cm, hm, p);
+    e = launch_chained(score_tc_kernel<kColsum, D, MASK>, grid, dim3(kTcThreads), smem, stream, qm, cm, hm, p);
     if (e != cudaSuccess) return e;
     dim3 cgrid((bv.max_cache + bv.max_chunk + 256 * kCombinePerThread - 1) / (256 * kCombinePerThread), mv.L * p.out_groups,
                bv.batch);
@@ -929,7 +970,9 @@ cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorVie
     p.merged = partial + (size_t)p.splits * kGroups * rows;
     p.work_prefix = (unsigned long long *)(p.merged + rows);
     p.score_parts = (float *)(p.merged + rows + plan_f2);
-    return mv.d == 64 ? launch_d<64>(ctx, qm, cm, hm, p, stream) : launch_d<128>(ctx, qm, cm, hm, p, stream);
+    if (bv.row_limit)  // causal query rows: the masked instantiation
+        return mv.d == 64 ? launch_d<64, true>(ctx, qm, cm, hm, p, stream) : launch_d<128, true>(ctx, qm, cm, hm, p, stream);
+    return mv.d == 64 ? launch_d<64, false>(ctx, qm, cm, hm, p, stream) : launch_d<128, false>(ctx, qm, cm, hm, p, stream);
 }
 
 }  // namespace finch
