@@ -31,7 +31,7 @@ UNIT = "tokens/s"
 FALLBACK_PEAK_GBS = 6650.0
 # DRAM bytes (read + write) of one full step from ncu, per configuration: captured on an 8-layer slice and scaled by
 # the unit count (profiles/step_kernels_c3_8layers.txt).  Must be set back to None whenever a kernel changes.
-TRAFFIC_BYTES = {"c3": 1016622080}
+TRAFFIC_BYTES = {"c3": 1021440000}
 MUFU_PER_CLK_PER_SM = 16   # exp2 results per clock per SM (4 per scheduler)
 
 
