@@ -67,6 +67,7 @@ class DocumentCompressor:
         self.kept_idx = torch.full((n_layers, self.G, total_cap), -1, dtype=torch.int32, device=device)
         self.cache_len = np.zeros(self.B, dtype=np.int32)       # host mirror of the device lengths
         self._ws = None
+        self._meta = {}
         self.steps = 0
 
     # the cache the next step will read
@@ -85,6 +86,7 @@ class DocumentCompressor:
     def reset(self) -> None:
         """Start a new batch of documents in the same buffers (empty caches)."""
         self.cache_len = np.zeros(self.B, dtype=np.int32)
+        self._bufs[0]["len"].zero_()
         self._cur = 0
         self.steps = 0
 
@@ -93,24 +95,49 @@ class DocumentCompressor:
             fb.finch_ctx_destroy(self.ctx)
             self.ctx = None
 
+    def _device_i32(self, a: np.ndarray):
+        """Device copy of a small int32 array, cached by content (offsets and budgets repeat from step to step)."""
+        key = a.tobytes()
+        t = self._meta.get(key)
+        if t is None:
+            if len(self._meta) > 256:
+                self._meta.clear()
+            t = self.torch.from_numpy(a.copy()).to(self.device)
+            self._meta[key] = t
+        return t
+
     def step(self, q, q_off: Sequence[int], chunk_k, chunk_v, chunk_pos, chunk_off: Sequence[int],
-             budget: Sequence[int], scores=None, prompt_self_lse=None) -> None:
-        """One finch_step: [cache ; chunk] -> the other cache.  Enqueues and returns."""
+             budget: Sequence[int], scores=None, prompt_self_lse=None, row_limit=None, row_norm=False) -> None:
+        """One finch_step: [cache ; chunk] -> the other cache.  Enqueues and returns.
+
+        The lengths the previous step wrote on the device are this step's cache lengths as they are: nothing comes
+        back to the host between steps, and the only host-to-device traffic is metadata that has not been seen yet."""
         torch = self.torch
         src, dst = self._bufs[self._cur], self._bufs[self._cur ^ 1]
-        budget = np.minimum(np.asarray(budget, dtype=np.int32), self.capacity)
-        batch = fb.make_batch(q_off, chunk_off, self.cache_off, self.cache_len, budget, self.device,
-                              prompt_self_lse=prompt_self_lse)
+        B = self.B
+        q_off = np.ascontiguousarray(q_off, dtype=np.int32)
+        chunk_off = np.ascontiguousarray(chunk_off, dtype=np.int32)
+        budget = np.minimum(np.asarray(budget, dtype=np.int32), self.capacity).astype(np.int32)
+        assert len(q_off) == len(chunk_off) == B + 1 and len(budget) == B
+        n_q, chunk_len = np.diff(q_off), np.diff(chunk_off)
+        n_cand = self.cache_len + chunk_len
+        mx = lambda a: int(a.max()) if len(a) else 0
+        c = fb.finch_batch(B, self._device_i32(q_off).data_ptr(), self._device_i32(chunk_off).data_ptr(),
+                           self._device_i32(self.cache_off).data_ptr(), src["len"].data_ptr(),
+                           self._device_i32(budget).data_ptr(), int(q_off[B]), int(chunk_off[B]), int(self.cache_off[B]),
+                           mx(n_q), mx(self.cache_len), mx(chunk_len), mx(np.minimum(budget, n_cand)),
+                           int(n_q.min()) if B else 0,
+                           prompt_self_lse.data_ptr() if prompt_self_lse is not None else None,
+                           row_limit.data_ptr() if row_limit is not None else None, int(bool(row_norm)))
+        batch = fb.Batch(None, None, None, None, None, c, prompt_self_lse, row_limit)
         need = fb.finch_workspace_bytes(self.ctx, batch)
         if self._ws is None or self._ws.numel() < need:
             self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
         fb.finch_step(self.ctx, q, src["k"], src["v"], src["pos"], chunk_k, chunk_v, chunk_pos, batch, dst["k"], dst["v"],
                       dst["pos"], self.kept_idx, dst["len"], scores, self._ws)
-        chunk_len = np.diff(np.asarray(chunk_off, dtype=np.int32))
-        self.cache_len = np.minimum(budget, self.cache_len + chunk_len).astype(np.int32)
+        self.cache_len = np.minimum(budget, n_cand).astype(np.int32)   # what the step writes to dst["len"]
         self._cur ^= 1
         self.steps += 1
-        self._last_batch = batch      # keeps the metadata tensors alive until the step has run
 
     def status(self) -> int:
         return fb.finch_device_status(self.ctx)
