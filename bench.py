@@ -6,13 +6,19 @@
 One "step" is one steady-state finch_step over all layers of the configuration (cache full, one new chunk).
 Prints ONE JSON line: candidate KV tokens/s (whole job), ms per step, the HBM roofline of the step, an end-to-end
 figure with host buffers, and the fp64 CPU oracle timed on a bounded sample of the same workload.
-With N > 1 (launched by torchrun) every rank runs an independent replica; there is no data-path collective.
+The timed region is BLOCKS blocks of K steps each (K = --steps), every block bracketed by a barrier and a device
+synchronisation; ms_per_step is the median block's time / K.  Steps alternate between two complete sets of input
+and output buffers.
+With N > 1 every rank runs an independent replica (no data-path collective): under torchrun the ranks come from the
+environment; started directly, `--gpus N` spawns the N ranks itself, one process per GPU.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -29,10 +35,35 @@ from paper_2408_00167_b200 import workloads as wl  # noqa: E402
 METRIC = "candidate_kv_tokens_per_sec"
 UNIT = "tokens/s"
 FALLBACK_PEAK_GBS = 6650.0
-# DRAM bytes (read + write) of one full step from ncu, per configuration: captured on an 8-layer slice and scaled by
-# the unit count (profiles/step_kernels_c3_8layers.txt).  Must be set back to None whenever a kernel changes.
-TRAFFIC_BYTES = {"c3": 1021440000}
-MUFU_PER_CLK_PER_SM = 16   # exp2 results per clock per SM (4 per scheduler)
+MUFU_PER_CLK_PER_SM = 16   # exp2 results per clock per SM (4 per scheduler); profiles/exp2_rate.txt
+BLOCKS = 25                # timed blocks of --steps steps each; the median block is reported
+BUFFER_SETS = 2            # complete input/output buffer sets the steps alternate between
+TRAFFIC_FILE = ROOT / "profiles" / "dram_traffic.txt"
+
+
+def kernel_sources_digest() -> str:
+    """SHA-256 over the CUDA sources of the library (names and contents): identifies the kernels a profile was
+    taken on, also where no git history is at hand."""
+    h = hashlib.sha256()
+    csrc = ROOT / "paper_2408_00167_b200" / "csrc"
+    for p in sorted(list(csrc.glob("*.cu")) + list(csrc.glob("*.cuh"))):
+        h.update(p.name.encode())
+        h.update(p.read_bytes())
+    return h.hexdigest()
+
+
+def recorded_traffic(config: str):
+    """DRAM bytes (read + write) of one full step of `config` as ncu counted them, from profiles/dram_traffic.txt --
+    or None when the file has no entry for the configuration or was captured on other kernel sources.
+    Line format:  <config> <bytes per step> <sha256 of the kernel sources> [# comment]"""
+    if not TRAFFIC_FILE.exists():
+        return None
+    digest = kernel_sources_digest()
+    for line in TRAFFIC_FILE.read_text().splitlines():
+        f = line.split("#")[0].split()
+        if len(f) >= 3 and f[0] == config and f[2] == digest:
+            return int(f[1])
+    return None
 
 
 def peak_hbm():
@@ -119,10 +150,38 @@ def aggregate_over_ranks(ms_local: float, tokens_local: int, world: int, backend
     return float(t.item()), int(n.item())
 
 
-def oracle_sample(cfg: wl.Config, target_s: float = 12.0, max_layers: int = 32):
+def launch_replicas(n: int, argv: list, extra_env: dict = None) -> int:
+    """Start n ranks of `argv` (a python command line without the interpreter) on this node, one process per GPU,
+    with RANK / LOCAL_RANK / WORLD_SIZE / MASTER_ADDR / MASTER_PORT set as torchrun would; rank 0 inherits stdout.
+    Waits for all of them; if one fails the others are terminated (by their own PIDs).  Returns the worst exit code."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    procs = []
+    for rank in range(n):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port), **(extra_env or {}))
+        procs.append(subprocess.Popen([sys.executable, *argv], env=env,
+                                      stdout=None if rank == 0 else subprocess.DEVNULL))
+    worst, pending = 0, set(range(n))
+    while pending:
+        for rank in sorted(pending):
+            rc = procs[rank].poll()
+            if rc is None:
+                continue
+            pending.discard(rank)
+            worst = max(worst, abs(rc))
+            if rc != 0:                      # a failed rank would leave the others waiting at a barrier
+                for other in pending:
+                    procs[other].terminate()
+        time.sleep(0.05)
+    return worst
+
+
+def oracle_sample(cfg: wl.Config, target_s: float = 12.0, max_layers: int = 32, threads: int = 0):
     """Time the fp64 oracle's whole step on whole layers of the same workload until about target_s of CPU work."""
     import oracle
-    threads = oracle.max_threads()
+    threads = threads or oracle.max_threads()
     total, layers_done, tokens = 0.0, 0, None
     while layers_done < min(max_layers, cfg.n_layers) and (layers_done == 0 or total < target_s):
         st = wl.steady_state(cfg, [layers_done])
@@ -143,7 +202,6 @@ def oracle_sample(cfg: wl.Config, target_s: float = 12.0, max_layers: int = 32):
 def run_ours(args, cfg: wl.Config):
     import torch
     import torch.distributed as dist
-    sys.path.insert(0, str(ROOT / "tests"))
     from paper_2408_00167_b200 import binding as fb
     from paper_2408_00167_b200 import build as fbuild
     rank, local_rank, world = dist_env()
@@ -168,7 +226,6 @@ def run_ours(args, cfg: wl.Config):
         t = t.pin_memory()
         return t.view(dt) if a.dtype == np.uint16 else t
     host = {k: pinned(st[k]) for k in ("q", "cache_k", "cache_v", "chunk_k", "chunk_v", "cache_pos", "chunk_pos")}
-    dev = {k: v.cuda(non_blocking=True) for k, v in host.items()}
     batch = fb.make_batch(st["q_off"], st["chunk_off"], st["cache_off"], st["cache_len"], st["budget"])
     c = batch.c
     ctx = fb.finch_ctx_create(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim,
@@ -176,27 +233,40 @@ def run_ours(args, cfg: wl.Config):
                               max_batch=cfg.batch, max_prompt=c.max_q, max_candidates=c.max_cache + c.max_chunk,
                               device=local_rank)
     G = cfg.n_groups
-    out_k, out_v = torch.empty_like(dev["cache_k"]), torch.empty_like(dev["cache_v"])
-    out_pos = torch.empty((cfg.n_layers, G, c.total_cache), dtype=torch.int32, device="cuda")
-    kept = torch.empty((cfg.n_layers, G, c.total_cache), dtype=torch.int32, device="cuda")
-    out_len = torch.empty(cfg.batch, dtype=torch.int32, device="cuda")
-    scores = torch.empty((cfg.n_layers, G, c.total_cache + c.total_chunk), dtype=torch.float32, device="cuda")
+
+    def buffer_set():
+        d = {k: v.cuda(non_blocking=True) for k, v in host.items()}
+        d["out_k"], d["out_v"] = torch.empty_like(d["cache_k"]), torch.empty_like(d["cache_v"])
+        d["out_pos"] = torch.empty((cfg.n_layers, G, c.total_cache), dtype=torch.int32, device="cuda")
+        d["kept"] = torch.empty((cfg.n_layers, G, c.total_cache), dtype=torch.int32, device="cuda")
+        d["out_len"] = torch.empty(cfg.batch, dtype=torch.int32, device="cuda")
+        d["scores"] = torch.empty((cfg.n_layers, G, c.total_cache + c.total_chunk), dtype=torch.float32, device="cuda")
+        return d
+    # consecutive steps work on different buffers: nothing a step reads or writes is left in L2 by the step before
+    sets = [buffer_set() for _ in range(BUFFER_SETS)]
+    dev = sets[0]
     ws = torch.empty(fb.finch_workspace_bytes(ctx, batch), dtype=torch.uint8, device="cuda")
-    kept_host = torch.empty_like(kept, device="cpu").pin_memory()
-    len_host = torch.empty_like(out_len, device="cpu").pin_memory()
+    kept_host = torch.empty_like(dev["kept"], device="cpu").pin_memory()
+    len_host = torch.empty_like(dev["out_len"], device="cpu").pin_memory()
+    turn = [0]
 
     def step():
-        fb.finch_step(ctx, dev["q"], dev["cache_k"], dev["cache_v"], dev["cache_pos"], dev["chunk_k"], dev["chunk_v"],
-                      dev["chunk_pos"], batch, out_k, out_v, out_pos, kept, out_len, scores, ws)
+        d = sets[turn[0] % BUFFER_SETS]
+        turn[0] += 1
+        fb.finch_step(ctx, d["q"], d["cache_k"], d["cache_v"], d["cache_pos"], d["chunk_k"], d["chunk_v"],
+                      d["chunk_pos"], batch, d["out_k"], d["out_v"], d["out_pos"], d["kept"], d["out_len"],
+                      d["scores"], ws)
 
     def step_e2e():
         # this step's inputs come from pinned host memory through the C ABI's host-buffer call; the cache is
         # carried on the device; the kept positions and lengths come back to the host
         fb.finch_step_host(ctx, host["q"], host["chunk_k"], host["chunk_v"], host["chunk_pos"], dev["q"],
                            dev["chunk_k"], dev["chunk_v"], dev["chunk_pos"], dev["cache_k"], dev["cache_v"],
-                           dev["cache_pos"], batch, out_k, out_v, out_pos, kept, out_len, kept_host, len_host, ws)
+                           dev["cache_pos"], batch, dev["out_k"], dev["out_v"], dev["out_pos"], dev["kept"],
+                           dev["out_len"], kept_host, len_host, ws)
 
     def timed(fn, n):
+        """n calls of fn between two events, with a barrier and a device synchronisation on both sides."""
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         if world > 1:
             dist.barrier()
@@ -215,28 +285,30 @@ def run_ours(args, cfg: wl.Config):
     assert fb.finch_device_status(ctx) == 0
     launches0 = fb.finch_launch_count(ctx)
     t_begin = time.time()
-    ms_local = timed(step, args.steps)
+    block_ms = [timed(step, args.steps) for _ in range(BLOCKS)]
     t_end = time.time()
-    launches = fb.finch_launch_count(ctx) - launches0
+    launches = (fb.finch_launch_count(ctx) - launches0) // BLOCKS       # per block of --steps steps
     assert fb.finch_device_status(ctx) == 0
+    ms_local = statistics.median(block_ms)
     ms, tokens = aggregate_over_ranks(ms_local, counts["tokens"], world, "nccl")
+    clocks = sampler.stop(t_begin, t_end)
 
     # per-phase durations (same kernels, called through the three separate entry points)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
     phase = np.zeros(3)
-    for _ in range(args.steps):
+    for i in range(args.steps):
+        d = sets[i % BUFFER_SETS]
         ev[0].record()
-        fb.finch_score(ctx, dev["q"], dev["cache_k"], dev["chunk_k"], batch, scores, None, ws)
+        fb.finch_score(ctx, d["q"], d["cache_k"], d["chunk_k"], batch, d["scores"], None, ws)
         ev[1].record()
-        fb.finch_select(ctx, scores, batch, kept, out_len)
+        fb.finch_select(ctx, d["scores"], batch, d["kept"], d["out_len"])
         ev[2].record()
-        fb.finch_compact(ctx, kept, out_len, dev["cache_k"], dev["cache_v"], dev["cache_pos"], dev["chunk_k"],
-                         dev["chunk_v"], dev["chunk_pos"], batch, out_k, out_v, out_pos)
+        fb.finch_compact(ctx, d["kept"], d["out_len"], d["cache_k"], d["cache_v"], d["cache_pos"], d["chunk_k"],
+                         d["chunk_v"], d["chunk_pos"], batch, d["out_k"], d["out_v"], d["out_pos"])
         ev[3].record()
         torch.cuda.synchronize()
         phase += [ev[i].elapsed_time(ev[i + 1]) for i in range(3)]
     phase /= args.steps
-    clocks = sampler.stop(t_begin, t_end)
 
     step_e2e()
     ms_e2e_local = timed(step_e2e, max(1, min(args.steps, 5)))
@@ -258,19 +330,25 @@ def run_ours(args, cfg: wl.Config):
     line = {
         "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "timing": {"blocks": BLOCKS, "steps_per_block": args.steps, "statistic": "median block / steps",
+                   "block_ms_min": min(block_ms), "block_ms_max": max(block_ms),
+                   # time x clock: comparable between runs that saw different SM clocks
+                   "kclk_per_step": ms_local * clocks["sm_mhz"] if clocks.get("sm_mhz") else None},
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic (seeded Gaussian / Student-t with planted keys)",
         "config": {"workload": f"{cfg.name}: {cfg.n_layers} layers x {cfg.n_q_heads}q/{cfg.n_kv_heads}kv heads, "
                                f"d{cfg.head_dim}, batch {cfg.batch}, {counts['tokens']} candidates per step, "
                                f"steady-state step (cache full)",
-                   "l2": "inputs larger than L2 (K+V+outputs per step exceed 126 MB)" if
-                   counts["contract_bytes"] > 2.5e8 else "working set fits L2 (latency-bound configuration)",
+                   "l2": (f"steps alternate between {BUFFER_SETS} complete buffer sets; " +
+                          ("inputs larger than L2 (K+V+outputs per step exceed 126 MB)" if
+                           counts["contract_bytes"] > 2.5e8 else "one set fits L2 (latency-bound configuration)")),
                    "replicas": "independent replicas, no collective"},
         "clocks": clocks,
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                 "d2h_bytes_per_step": int(d2h), "ms_per_step": ms_e2e},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": TRAFFIC_BYTES.get(cfg.name) if cfg.n_layers == wl.CONFIGS[cfg.name].n_layers else None,
+                     # ncu's DRAM bytes of one step, only if they were captured on exactly these kernel sources
+                     "traffic": recorded_traffic(cfg.name) if cfg.n_layers == wl.CONFIGS[cfg.name].n_layers else None,
                      "peak_kind": f"of {peak_kind}",
                      "algorithmic_bytes_per_step": counts["contract_bytes"],
                      "kernel": "whole step (score + select + compact launches)"},
@@ -356,7 +434,7 @@ def run_reference(args, cfg: wl.Config):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="c3", choices=sorted(wl.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -367,6 +445,9 @@ def main():
     ap.add_argument("--group-mode", type=int, default=-1, choices=[-1, 0, 1],
                     help="selection groups of the document loop: 0 per KV head, 1 per layer (-1: the configuration's)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        # started directly rather than by torchrun: be the launcher of the N replicas
+        sys.exit(launch_replicas(args.gpus, [str(Path(__file__).resolve()), *sys.argv[1:]]))
     cfg = wl.CONFIGS[args.config]
     if args.layers > 0:
         cfg = wl.scaled(cfg, n_layers=min(args.layers, cfg.n_layers))
@@ -377,6 +458,9 @@ def main():
         rank, _, world = dist_env()
         if line is not None and world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"], _ = oracle_sample(cfg)
+            one, _ = oracle_sample(cfg, target_s=0.0, max_layers=1, threads=1)
+            line["cpu_baseline"]["single_thread"] = {"value": one["value"], "unit": UNIT, "cores": 1,
+                                                     "sample": one["sample"]}
     if line is not None:
         print(json.dumps(line), flush=True)
 

@@ -116,7 +116,6 @@ typedef struct {
     const int32_t *cache_len, *budget;            /* device, [batch]; budget[b] = r, at most the capacity     */
     int32_t total_q, total_chunk, total_cache;    /* host copies of q_off[batch], chunk_off[batch], cache_off[batch] */
     int32_t max_q, max_cache, max_chunk, max_budget; /* host upper bounds over the requests (grid sizing)      */
-    int32_t min_q;                                /* host lower bound of the prompt lengths; 0 when unknown    */
     /* Optional (NULL = absent), device, [n_layers][n_q_heads][total_q] fp32, natural log: for every prompt row the
      * log-sum-exp of its scaled logits against the keys it attends to besides the candidates -- in the paper's
      * full forward pass the prompt's own (causally visible) keys, "N = m + n^que + c" (Method, bullet "Extract

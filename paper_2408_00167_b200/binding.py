@@ -52,7 +52,7 @@ class finch_batch(C.Structure):
                 ("cache_len", C.c_void_p), ("budget", C.c_void_p), ("total_q", C.c_int32),
                 ("total_chunk", C.c_int32), ("total_cache", C.c_int32), ("max_q", C.c_int32),
                 ("max_cache", C.c_int32), ("max_chunk", C.c_int32), ("max_budget", C.c_int32),
-                ("min_q", C.c_int32), ("prompt_self_lse", C.c_void_p), ("row_limit", C.c_void_p),
+                ("prompt_self_lse", C.c_void_p), ("row_limit", C.c_void_p),
                 ("row_norm", C.c_int32)]
 
 
@@ -150,7 +150,6 @@ def make_batch(q_off: Sequence[int], chunk_off: Sequence[int], cache_off: Sequen
     n_cand = h[3] + diff(h[1])
     cb = finch_batch(B, *[x.data_ptr() for x in d], int(h[0][B]), int(h[1][B]), int(h[2][B]),
                      mx(diff(h[0])), mx(h[3]), mx(diff(h[1])), mx(np.minimum(h[4], n_cand)) if B else 0,
-                     int(diff(h[0]).min()) if B else 0,
                      prompt_self_lse.data_ptr() if prompt_self_lse is not None else None,
                      row_limit.data_ptr() if row_limit is not None else None, int(bool(row_norm)))
     return Batch(*d, cb, prompt_self_lse, row_limit)

@@ -4,6 +4,7 @@
 #include <new>
 #include <string.h>
 
+#include <atomic>
 #include <vector>
 
 #include "finch_internal.cuh"
@@ -33,7 +34,6 @@ finch_status check_batch(const finch_ctx *ctx, const finch_batch *b) {
     if (!ctx || !b) return FINCH_ERR_INVALID_ARG;
     if (b->batch < 0 || b->batch > ctx->cfg.max_batch) return FINCH_ERR_INVALID_ARG;
     if (b->total_q < 0 || b->total_chunk < 0 || b->total_cache < 0) return FINCH_ERR_INVALID_ARG;
-    if (b->min_q < 0 || b->min_q > b->max_q) return FINCH_ERR_INVALID_ARG;
     if (b->max_q < 0 || b->max_cache < 0 || b->max_chunk < 0 || b->max_budget < 0) return FINCH_ERR_INVALID_ARG;
     if (b->max_q > ctx->cfg.max_prompt) return FINCH_ERR_INVALID_ARG;
     if ((int64_t)b->max_cache + b->max_chunk > ctx->cfg.max_candidates) return FINCH_ERR_INVALID_ARG;
@@ -68,7 +68,30 @@ WsLayout ws_layout(const finch_ctx *ctx, const finch_batch *b) {
 
 finch_status cuda_status(cudaError_t e) { return e == cudaSuccess ? FINCH_OK : FINCH_ERR_CUDA; }
 
-bool same_base(const finch_tensor *a, const finch_tensor *b) { return a && b && a->ptr && a->ptr == b->ptr; }
+// Do two [layers][heads][tokens][head_dim] views share a byte?  Their byte extents are compared; extents that
+// intersect are still disjoint when both views have the same strides, whole rows as their head and layer strides,
+// and base pointers that differ by a shift which keeps every row of one between the rows of the other (K and V
+// interleaved in one buffer).  Anything else that intersects counts as an overlap.
+bool views_overlap(const finch_ctx *ctx, const finch_tensor *a, int64_t a_tokens, const finch_tensor *b,
+                   int64_t b_tokens) {
+    if (!a || !b || !a->ptr || !b->ptr || a_tokens <= 0 || b_tokens <= 0) return false;
+    const ModelView &mv = ctx->model;
+    const int64_t e = mv.elem_bytes, row = (int64_t)mv.d * e;
+    auto extent = [&](const finch_tensor *t, int64_t tokens) {
+        return ((int64_t)(mv.L - 1) * t->stride_layer + (int64_t)(mv.Hkv - 1) * t->stride_head +
+                (tokens - 1) * t->stride_tok) * e + row;
+    };
+    const uintptr_t a0 = (uintptr_t)a->ptr, b0 = (uintptr_t)b->ptr;
+    const uintptr_t a1 = a0 + (uintptr_t)extent(a, a_tokens), b1 = b0 + (uintptr_t)extent(b, b_tokens);
+    if (a1 <= b0 || b1 <= a0) return false;
+    const int64_t pitch = a->stride_tok * e;
+    if (a->stride_tok == b->stride_tok && a->stride_head == b->stride_head && a->stride_layer == b->stride_layer &&
+        a->stride_head % a->stride_tok == 0 && a->stride_layer % a->stride_tok == 0 && pitch >= 2 * row) {
+        const int64_t shift = (int64_t)((a0 > b0 ? a0 - b0 : b0 - a0) % (uintptr_t)pitch);
+        if (shift >= row && shift <= pitch - row) return false;  // rows of one lie in the gaps of the other
+    }
+    return true;
+}
 
 finch_status validate_score(const finch_ctx *ctx, const finch_tensor *q, const finch_tensor *cache_k,
                             const finch_tensor *chunk_k, const finch_batch *batch) {
@@ -99,12 +122,15 @@ finch_status validate_compact(const finch_ctx *ctx, const int32_t *kept_idx, con
     if (!no_chunk && !chunk_pos) return FINCH_ERR_INVALID_ARG;
     if (batch->max_cache > 0 && !cache_pos) return FINCH_ERR_INVALID_ARG;
     if (batch->batch > 0 && !out_len) return FINCH_ERR_INVALID_ARG;
+    // the gather runs in parallel: an output row that shares bytes with any input row, or with the other output,
+    // would race
     const finch_tensor *outs[2] = {out_k, out_v};
     const finch_tensor *ins[4] = {cache_k, cache_v, chunk_k, chunk_v};
+    const int64_t in_tokens[4] = {batch->total_cache, batch->total_cache, batch->total_chunk, batch->total_chunk};
     for (auto o : outs)
-        for (auto i : ins)
-            if (same_base(o, i)) return FINCH_ERR_INVALID_ARG;
-    if (same_base(out_k, out_v)) return FINCH_ERR_INVALID_ARG;
+        for (int i = 0; i < 4; ++i)
+            if (views_overlap(ctx, o, batch->total_cache, ins[i], in_tokens[i])) return FINCH_ERR_INVALID_ARG;
+    if (views_overlap(ctx, out_k, batch->total_cache, out_v, batch->total_cache)) return FINCH_ERR_INVALID_ARG;
     return FINCH_OK;
 }
 
@@ -118,11 +144,11 @@ cudaError_t run_score(const Ctx &ctx, const TensorView &q, const TensorView &cac
                       const BatchView &bv, float *scores, float2 *scratch, size_t scratch_capacity, float *row_lse,
                       cudaStream_t stream) {
     if (score_tc_supported(ctx)) {
-        const cudaError_t e = launch_score_tc(ctx, q, cache_k, chunk_k, bv, scores, scratch, scratch_capacity, row_lse,
-                                              /*min_q=*/1, stream);
+        const cudaError_t e =
+            launch_score_tc(ctx, q, cache_k, chunk_k, bv, scores, scratch, scratch_capacity, row_lse, stream);
         if (e != cudaErrorNotSupported) return e;
     }
-    return launch_score_simt(ctx, q, cache_k, chunk_k, bv, scores, scratch, row_lse, INT_MAX, stream);
+    return launch_score_simt(ctx, q, cache_k, chunk_k, bv, scores, scratch, row_lse, stream);
 }
 
 }  // namespace finch
@@ -193,6 +219,15 @@ finch_status finch_ctx_create(const finch_config *cfg, finch_ctx **out) {
             return FINCH_ERR_UNSUPPORTED;
         }
         ctx->sm_count = prop.multiProcessorCount;
+        // the context's device is made current only while its resources are created; the caller's comes back after
+        int caller_device = -1;
+        if (cudaGetDevice(&caller_device) != cudaSuccess) caller_device = -1;
+        struct Restore {
+            int dev;
+            ~Restore() {
+                if (dev >= 0) (void)cudaSetDevice(dev);
+            }
+        } restore{caller_device == cfg->device ? -1 : caller_device};
         if (cudaSetDevice(cfg->device) != cudaSuccess || cudaMalloc(&ctx->d_status, sizeof(int)) != cudaSuccess) {
             (void)cudaGetLastError();
             delete ctx;
@@ -440,26 +475,28 @@ constexpr size_t kStaticRows = size_t(1) << 20;  // prompt rows (layers x query 
 static __device__ __align__(256) float2 g_static_row_stats[kStaticRows];
 
 constexpr int kMaxDevices = 64;
-float2 *g_static_ptr[kMaxDevices] = {};  // device address of the array on each device, filled on first use
+// device address of the array on each device, filled on first use; contexts on different host threads share it
+std::atomic<float2 *> g_static_ptr[kMaxDevices];
 
 // In host code the array's name is only a handle; its device address has to be asked for, once per device, with
-// that device current.
+// that device current.  The current device is checked on every call: the address belongs to one GPU, and kernels
+// launched with another device current would dereference it there.
 finch_status static_scratch(int device, float2 **out) {
     if (device < 0 || device >= kMaxDevices) return FINCH_ERR_UNSUPPORTED;
-    if (!g_static_ptr[device]) {
-        int current = -1;
-        if (cudaGetDevice(&current) != cudaSuccess || current != device) {
-            (void)cudaGetLastError();
-            return FINCH_ERR_INVALID_ARG;  // the context's device must be the current one
-        }
-        float2 *p = nullptr;
+    int current = -1;
+    if (cudaGetDevice(&current) != cudaSuccess || current != device) {
+        (void)cudaGetLastError();
+        return FINCH_ERR_INVALID_ARG;  // the context's device must be the current one
+    }
+    float2 *p = g_static_ptr[device].load(std::memory_order_acquire);
+    if (!p) {
         if (cudaGetSymbolAddress((void **)&p, g_static_row_stats) != cudaSuccess || !p) {
             (void)cudaGetLastError();
             return FINCH_ERR_CUDA;
         }
-        g_static_ptr[device] = p;
+        g_static_ptr[device].store(p, std::memory_order_release);  // every thread resolves the same address
     }
-    *out = g_static_ptr[device];
+    *out = p;
     return FINCH_OK;
 }
 

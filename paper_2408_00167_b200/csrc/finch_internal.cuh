@@ -20,7 +20,6 @@ struct BatchView {
     const int *q_off, *chunk_off, *cache_off, *cache_len, *budget;
     int total_q, total_chunk, total_cache;
     int max_q, max_cache, max_chunk, max_budget;
-    int min_q;
     const float *self_lse;  // optional extra softmax-denominator term per prompt row (natural log), or null
     const int *row_limit;   // optional visible-candidate count per query row [total_q], or null
     int row_norm;           // scale a row's weights by the fraction of the candidates it sees
@@ -61,7 +60,7 @@ inline TensorView view_of(const finch_tensor *t) {
 inline BatchView view_of(const finch_batch *b) {
     return BatchView{b->batch,       b->q_off,       b->chunk_off, b->cache_off, b->cache_len, b->budget,    b->total_q,
                      b->total_chunk, b->total_cache, b->max_q,     b->max_cache, b->max_chunk, b->max_budget,
-                     b->min_q,       b->prompt_self_lse, b->row_limit, b->row_norm};
+                     b->prompt_self_lse, b->row_limit, b->row_norm};
 }
 
 constexpr float kLog2e = 1.4426950408889634f;
@@ -88,8 +87,10 @@ __device__ __forceinline__ UnitInfo unit_info(const ModelView &mv, const BatchVi
     u.c = bv.cache_len[b];
     u.m = bv.chunk_off[b + 1] - u.chunk0;
     u.N = u.c + u.m;
+    // lengths within the host bounds, and every region inside its packed tensor (the offsets come from device memory)
     u.ok = u.n_q >= 0 && u.n_q <= bv.max_q && u.c >= 0 && u.c <= bv.max_cache && u.m >= 0 && u.m <= bv.max_chunk &&
-           u.c <= u.cap;
+           u.c <= u.cap && u.q0 >= 0 && u.q0 <= bv.total_q - u.n_q && u.cache0 >= 0 && u.cap >= 0 &&
+           u.cache0 <= bv.total_cache - u.cap && u.chunk0 >= 0 && u.chunk0 <= bv.total_chunk - u.m;
     return u;
 }
 
@@ -125,16 +126,16 @@ cudaError_t launch_chained(void (*kernel)(Params...), dim3 grid, dim3 block, siz
 // warp-level dot-product scoring (any dtype, any prompt length).  row_stats [L][Hq][total_q] is scratch that holds
 // (max base-2 logit, 1 / sum of exp2) per prompt row; row_lse (nullable) is the caller-visible natural-log copy.
 cudaError_t launch_score_simt(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
-                              const BatchView &bv, float *scores, float2 *row_stats, float *row_lse, int nq_below,
+                              const BatchView &bv, float *scores, float2 *row_stats, float *row_lse,
                               cudaStream_t stream);
 
-// tensor-core scoring (bf16, head_dim 64 or 128, either group mode) for requests with n_q >= min_q.  The scratch
+// tensor-core scoring (bf16, head_dim 64 or 128, either group mode).  The scratch
 // holds one float2 per prompt row and key split; up to kScoreMaxSplits splits are used when it is large enough.
 constexpr int kScoreMaxSplits = 8;
 bool score_tc_supported(const Ctx &ctx);
 cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
                             const BatchView &bv, float *scores, float2 *partial, size_t partial_capacity,
-                            float *row_lse, int min_q, cudaStream_t stream);
+                            float *row_lse, cudaStream_t stream);
 
 // scoring dispatch shared by finch_score, finch_score_static and finch_step; `scratch` holds scratch_capacity
 // float2 entries, at least one per prompt row (n_layers * n_q_heads * total_q)

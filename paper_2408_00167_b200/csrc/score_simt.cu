@@ -78,7 +78,7 @@ __device__ __forceinline__ void fma_slice(float (&acc)[4][4], const float (*qs)[
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 lse_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, TensorView chunk_k, float2 *row_stats,
-         float *row_lse, int *status, int nq_below) {
+         float *row_lse, int *status) {
     __shared__ float qs[kTile][kSlice + 1];
     __shared__ float ks[kTile][kSlice + 1];
     const UnitInfo u = unit_info(mv, bv, blockIdx.y, blockIdx.z);
@@ -86,7 +86,7 @@ lse_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, TensorVie
         if (threadIdx.x == 0) atomicOr(status, FINCH_DEV_BAD_BATCH);
         return;
     }
-    if (u.N == 0 || u.n_q >= nq_below) return;  // longer prompts belong to the tensor-core path
+    if (u.N == 0) return;
     const int row_blocks = (bv.max_q + kTile - 1) / kTile;
     const int hh = blockIdx.x / row_blocks, p0 = (blockIdx.x % row_blocks) * kTile;
     if (p0 >= u.n_q) return;
@@ -167,7 +167,7 @@ lse_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, TensorVie
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 colsum_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, TensorView chunk_k,
-            const float2 *row_stats, float *scores, int *status, int nq_below) {
+            const float2 *row_stats, float *scores, int *status) {
     __shared__ float qs[kTile][kSlice + 1];
     __shared__ float ks[kTile][kSlice + 1];
     __shared__ float red[16][kTile];
@@ -177,7 +177,7 @@ colsum_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, Tensor
         return;
     }
     const int j0 = blockIdx.x * kTile;
-    if (j0 >= u.N || u.n_q >= nq_below) return;
+    if (j0 >= u.N) return;
     const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
     const float scale2 = mv.scale * kLog2e;
 
@@ -221,7 +221,7 @@ colsum_simt(ModelView mv, BatchView bv, TensorView q, TensorView cache_k, Tensor
 
 template <typename T>
 cudaError_t launch_t(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
-                     const BatchView &bv, float *scores, float2 *row_stats, float *row_lse, int nq_below,
+                     const BatchView &bv, float *scores, float2 *row_stats, float *row_lse,
                      cudaStream_t stream) {
     const ModelView &mv = ctx.model;
     const int units = mv.L * mv.G;
@@ -229,9 +229,9 @@ cudaError_t launch_t(const Ctx &ctx, const TensorView &q, const TensorView &cach
     const int key_tiles = (bv.max_cache + bv.max_chunk + kTile - 1) / kTile;
     if (units == 0 || bv.batch == 0 || row_blocks == 0 || key_tiles == 0) return cudaSuccess;
     dim3 g1(row_blocks * mv.hpg, units, bv.batch);
-    lse_simt<T><<<g1, kThreads, 0, stream>>>(mv, bv, q, cache_k, chunk_k, row_stats, row_lse, ctx.d_status, nq_below);
+    lse_simt<T><<<g1, kThreads, 0, stream>>>(mv, bv, q, cache_k, chunk_k, row_stats, row_lse, ctx.d_status);
     dim3 g2(key_tiles, units, bv.batch);
-    colsum_simt<T><<<g2, kThreads, 0, stream>>>(mv, bv, q, cache_k, chunk_k, row_stats, scores, ctx.d_status, nq_below);
+    colsum_simt<T><<<g2, kThreads, 0, stream>>>(mv, bv, q, cache_k, chunk_k, row_stats, scores, ctx.d_status);
     ctx.launches += 2;
     return cudaGetLastError();
 }
@@ -239,11 +239,11 @@ cudaError_t launch_t(const Ctx &ctx, const TensorView &q, const TensorView &cach
 }  // namespace
 
 cudaError_t launch_score_simt(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
-                              const BatchView &bv, float *scores, float2 *row_stats, float *row_lse, int nq_below,
+                              const BatchView &bv, float *scores, float2 *row_stats, float *row_lse,
                               cudaStream_t stream) {
     if (ctx.cfg.dtype == FINCH_F32)
-        return launch_t<float>(ctx, q, cache_k, chunk_k, bv, scores, row_stats, row_lse, nq_below, stream);
-    return launch_t<__nv_bfloat16>(ctx, q, cache_k, chunk_k, bv, scores, row_stats, row_lse, nq_below, stream);
+        return launch_t<float>(ctx, q, cache_k, chunk_k, bv, scores, row_stats, row_lse, stream);
+    return launch_t<__nv_bfloat16>(ctx, q, cache_k, chunk_k, bv, scores, row_stats, row_lse, stream);
 }
 
 }  // namespace finch

@@ -53,7 +53,6 @@ struct TcParams {
     float *scores;
     float *score_parts;  // [kGroups][L][G][total_cand] per-group partial column sums
     int *status;
-    int min_q;         // requests with fewer prompt rows are left to the warp-level path
     int splits;        // key splits per unit (grid x)
     int stages;        // key-tile ring depth that fits beside the resident queries
     int q_tiles;       // query tiles resident at a time (1..4), sized from the batch's longest prompt
@@ -311,7 +310,7 @@ __device__ __forceinline__ Item walk_item(Walk &k, const TcParams &p, bool repor
     if (k.req.b != k.b) {
         k.req = unit_info(p.mv, p.bv, 0, k.b);
         const UnitInfo &u = k.req;
-        k.req_run = u.ok && u.n_q >= p.min_q && u.N > 0;
+        k.req_run = u.ok && u.n_q > 0 && u.N > 0;
         k.k_tiles = n_key_tiles(u);
         k.tps = (k.k_tiles + p.splits - 1) / p.splits;  // key tiles per split
         k.sbq = (u.n_q + kSub - 1) / kSub;              // sub-blocks per query head
@@ -692,7 +691,7 @@ plan_items_kernel(TcParams p, int *bounds, int n_ctas) {
         unsigned long long cost = 0;
         if (b < bv.batch) {
             const UnitInfo u = unit_info(mv, bv, 0, b);
-            if (u.ok && u.n_q >= p.min_q && u.N > 0) {
+            if (u.ok && u.n_q > 0 && u.N > 0) {
                 const int sb = mv.hpg * ((u.n_q + kSub - 1) / kSub);
                 // key tiles of one split x query tiles, plus a little for the item's fixed costs
                 cost = ipr * (unsigned long long)((n_key_tiles(u) + p.splits - 1) / p.splits * ((sb + 1) / 2) + 2);
@@ -746,7 +745,7 @@ merge_stats_kernel(TcParams p) {
     dependency_wait();
     const int h = blockIdx.y % mv.Hq, l = blockIdx.y / mv.Hq;
     const UnitInfo u = unit_info(mv, bv, l * mv.G + h / mv.hpg, blockIdx.z);
-    if (!u.ok || u.n_q < p.min_q || u.N == 0) return;
+    if (!u.ok || u.n_q == 0 || u.N == 0) return;
     const int pr = blockIdx.x * 128 + threadIdx.x;
     if (pr >= u.n_q) return;
     const int k_tiles = n_key_tiles(u);
@@ -811,7 +810,7 @@ combine_scores_kernel(TcParams p) {
     dependency_wait();  // many waves of small CTAs: the next kernel's CTAs must not take their slots early
     const int l = blockIdx.y / p.out_groups, og = blockIdx.y % p.out_groups;
     const UnitInfo u = unit_info(mv, bv, l * mv.G + og * p.units_per_group, blockIdx.z);
-    if (!u.ok || (u.n_q > 0 && u.n_q < p.min_q)) return;
+    if (!u.ok) return;
     const int64_t cand = (int64_t)bv.total_cache + bv.total_chunk;
     const int64_t gstride = (int64_t)mv.L * mv.G * cand;
     // four keys per thread, 256 apart: every load is coalesced and a thread has up to 16 of them in flight
@@ -939,7 +938,7 @@ bool score_tc_supported(const Ctx &ctx) {
 // to the TMA unit; the caller then uses the warp-level path for every request.
 cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
                             const BatchView &bv, float *scores, float2 *partial, size_t partial_capacity,
-                            float *row_lse, int min_q, cudaStream_t stream) {
+                            float *row_lse, cudaStream_t stream) {
     // Scoring works per KV head whatever the selection groups are: a query head only ever meets its own KV head's
     // keys.  With one selection group per layer the heads' column sums are added when the parts are combined.
     ModelView mv = ctx.model;
@@ -964,7 +963,7 @@ cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorVie
     const int key_tiles = (bv.max_cache + kRows - 1) / kRows + (bv.max_chunk + kRows - 1) / kRows;
     const int max_splits =
         (int)min((size_t)kScoreMaxSplits, ((partial_capacity - parts_f2 - plan_f2) / rows - 1) / kGroups);
-    TcParams p{mv, bv, partial, nullptr, row_lse, scores, nullptr, ctx.d_status, min_q, 1, 2, 1, 0, nullptr, nullptr,
+    TcParams p{mv, bv, partial, nullptr, row_lse, scores, nullptr, ctx.d_status, 1, 2, 1, 0, nullptr, nullptr,
                ctx.model.G, ctx.model.kvpg};
     p.splits = choose_splits(mv.L * mv.G * bv.batch, key_tiles, ctx.sm_count > 0 ? ctx.sm_count : 148, max_splits);
     p.merged = partial + (size_t)p.splits * kGroups * rows;

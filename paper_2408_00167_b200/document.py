@@ -4,7 +4,9 @@
 against the prompt, keeps `budget` candidates and carries them to the next step ("Selection of top r position",
 "Managing the Cache").  This module only orchestrates: two caches on the device that swap roles each step, the batch
 metadata, and the budget schedule.  Every step is one finch_step call; nothing is computed here, and the loop never
-waits for the device (the lengths a step will produce are known on the host: out_len = min(budget, cache + chunk)).
+waits for the device: the lengths a step will produce are known on the host (out_len = min(budget, cache + chunk))
+and kept in a host mirror.  The mirror is only a prediction -- a step the device refused (status word set) writes
+length 0 -- so `verify` compares it with the device at the end of a document, and `reset` / `close` call it.
 """
 from __future__ import annotations
 
@@ -69,6 +71,7 @@ class DocumentCompressor:
         self._ws = None
         self._meta = {}
         self.steps = 0
+        self._unverified = 0    # steps enqueued since the device was last compared with the host mirror
 
     # the cache the next step will read
     @property
@@ -83,17 +86,37 @@ class DocumentCompressor:
     def cache_pos(self):
         return self._bufs[self._cur]["pos"]
 
+    def verify(self) -> None:
+        """Wait for the steps enqueued so far and check them: raises RuntimeError when the device status word is set
+        or when the lengths on the device differ from the host mirror the later steps were sized with."""
+        if self._unverified == 0:
+            return
+        self._unverified = 0
+        word = fb.finch_device_status(self.ctx)            # synchronises the stream
+        dev_len = self._bufs[self._cur]["len"][:self.B].cpu().numpy()
+        if word != 0:
+            raise RuntimeError(f"document loop: device status word {word:#x} after {self.steps} steps "
+                               f"(lengths on the device {dev_len.tolist()}, expected {self.cache_len.tolist()})")
+        if not np.array_equal(dev_len, self.cache_len):
+            raise RuntimeError(f"document loop: cache lengths on the device {dev_len.tolist()} differ from the "
+                               f"host mirror {self.cache_len.tolist()} after {self.steps} steps")
+
     def reset(self) -> None:
-        """Start a new batch of documents in the same buffers (empty caches)."""
+        """Start a new batch of documents in the same buffers (empty caches).  Checks the finished one first."""
+        self.verify()
         self.cache_len = np.zeros(self.B, dtype=np.int32)
         self._bufs[0]["len"].zero_()
         self._cur = 0
         self.steps = 0
 
     def close(self) -> None:
+        """Check the steps still unverified, then free the context (the check's error, if any, is raised after)."""
         if self.ctx:
-            fb.finch_ctx_destroy(self.ctx)
-            self.ctx = None
+            try:
+                self.verify()
+            finally:
+                fb.finch_ctx_destroy(self.ctx)
+                self.ctx = None
 
     def _device_i32(self, a: np.ndarray):
         """Device copy of a small int32 array, cached by content (offsets and budgets repeat from step to step)."""
@@ -126,7 +149,6 @@ class DocumentCompressor:
                            self._device_i32(self.cache_off).data_ptr(), src["len"].data_ptr(),
                            self._device_i32(budget).data_ptr(), int(q_off[B]), int(chunk_off[B]), int(self.cache_off[B]),
                            mx(n_q), mx(self.cache_len), mx(chunk_len), mx(np.minimum(budget, n_cand)),
-                           int(n_q.min()) if B else 0,
                            prompt_self_lse.data_ptr() if prompt_self_lse is not None else None,
                            row_limit.data_ptr() if row_limit is not None else None, int(bool(row_norm)))
         batch = fb.Batch(None, None, None, None, None, c, prompt_self_lse, row_limit)
@@ -138,6 +160,8 @@ class DocumentCompressor:
         self.cache_len = np.minimum(budget, n_cand).astype(np.int32)   # what the step writes to dst["len"]
         self._cur ^= 1
         self.steps += 1
+        self._unverified += 1
 
     def status(self) -> int:
+        """Wait for the stream and return (and clear) the device status word; 0 = clean."""
         return fb.finch_device_status(self.ctx)

@@ -13,6 +13,14 @@ from paper_2408_00167_b200 import workloads as wl
 
 REL_TOL, ABS_TOL = 1e-3, 1e-5   # per-key score tolerance for bf16/fp32 inputs with fp32 accumulation
 
+# Every output buffer starts out filled with a value the kernels never produce, and sits between two guard zones
+# of GUARD elements holding the same value: whatever is still there afterwards was not written.
+GUARD = 4096
+SENTINEL_I32 = -1          # kept_idx, out_pos
+SENTINEL_LEN = -7          # out_len
+SENTINEL_BF16 = 0x7FC5     # a NaN bit pattern no rounding produces (out_k / out_v rows, bf16 storage)
+SENTINEL_F32 = 0x7FC00005  # the same for fp32 storage (scores and row_lse use it as well)
+
 
 def to_device(a: np.ndarray, dtype: str, device="cuda"):
     """Storage bit patterns (float32 or uint16-as-bf16) -> torch tensor of the matching dtype on the device."""
@@ -59,15 +67,32 @@ class GpuStep:
         self.cache_pos = torch.from_numpy(np.ascontiguousarray(st["cache_pos"], dtype=np.int32)).to(device)
         self.chunk_pos = torch.from_numpy(np.ascontiguousarray(st["chunk_pos"], dtype=np.int32)).to(device)
         total_cache, total_cand = c.total_cache, c.total_cache + c.total_chunk
-        self.out_k = torch.zeros_like(self.cache_k)
-        self.out_v = torch.zeros_like(self.cache_v)
-        self.out_pos = torch.full((n_layers, self.G, total_cache), -1, dtype=torch.int32, device=device)
-        self.kept_idx = torch.full((n_layers, self.G, total_cache), -1, dtype=torch.int32, device=device)
-        self.out_len = torch.full((max(B, 1),), -7, dtype=torch.int32, device=device)
-        self.scores = torch.full((n_layers, self.G, total_cand), float("nan"), dtype=torch.float32, device=device)
-        self.row_lse = torch.full((n_layers, cfg.n_q_heads, c.total_q), float("nan"), dtype=torch.float32,
-                                  device=device)
+        self._guarded = []      # (flat integer tensor with the guard zones, sentinel) of every output buffer
+        store = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+        store_bits = SENTINEL_F32 if cfg.dtype == "f32" else SENTINEL_BF16
+        self.out_k = self._output(self.cache_k.shape, store, store_bits)
+        self.out_v = self._output(self.cache_v.shape, store, store_bits)
+        self.out_pos = self._output((n_layers, self.G, total_cache), torch.int32, SENTINEL_I32)
+        self.kept_idx = self._output((n_layers, self.G, total_cache), torch.int32, SENTINEL_I32)
+        self.out_len = self._output((max(B, 1),), torch.int32, SENTINEL_LEN)
+        self.scores = self._output((n_layers, self.G, total_cand), torch.float32, SENTINEL_F32)
+        self.row_lse = self._output((n_layers, cfg.n_q_heads, c.total_q), torch.float32, SENTINEL_F32)
         self.ws = torch.empty(fb.finch_workspace_bytes(self.ctx, self.batch), dtype=torch.uint8, device=device)
+
+    def _output(self, shape, dtype, sentinel: int):
+        """A contiguous output tensor of `shape`, sentinel-filled, with a guard zone of GUARD elements on each side."""
+        import torch
+        bits = {torch.float32: torch.int32, torch.bfloat16: torch.int16, torch.int32: torch.int32}[dtype]
+        n = int(np.prod(shape))
+        signed = sentinel - (1 << 16) if bits == torch.int16 and sentinel >= (1 << 15) else sentinel
+        flat = torch.full((n + 2 * GUARD,), signed, dtype=bits, device=self.device)
+        self._guarded.append((flat, n, signed))
+        return flat[GUARD:GUARD + n].view(dtype).view(*shape)
+
+    def guards_intact(self) -> bool:
+        """True when no kernel wrote before the start or past the end of any output buffer."""
+        return all(bool((flat[:GUARD] == s).all()) and bool((flat[GUARD + n:] == s).all())
+                   for flat, n, s in self._guarded)
 
     def close(self):
         fb.finch_ctx_destroy(self.ctx)
@@ -90,10 +115,13 @@ class GpuStep:
         return fb.finch_device_status(self.ctx)
 
     def results(self) -> dict:
+        """Host copies of the outputs.  `sentinels` tells check_parity that everything outside the valid regions
+        must still hold the initial fill; the guard zones around the buffers are checked right here."""
+        assert self.guards_intact(), "a kernel wrote outside an output buffer"
         return dict(scores=self.scores.cpu().numpy(), kept_idx=self.kept_idx.cpu().numpy(),
                     out_len=self.out_len.cpu().numpy(), out_pos=self.out_pos.cpu().numpy(),
                     out_k=to_host(self.out_k, self.dtype), out_v=to_host(self.out_v, self.dtype),
-                    row_lse=self.row_lse.cpu().numpy())
+                    row_lse=self.row_lse.cpu().numpy(), sentinels=True)
 
 
 def oracle_scores(cfg: wl.Config, st: dict, group_mode=None, scale=None, threads=8, want_lse=False,
@@ -114,6 +142,9 @@ def check_parity(cfg: wl.Config, st: dict, res: dict, ref_scores: np.ndarray, gr
           is exactly r' and the indices strictly increase (tau = the oracle's r'-th largest score)
     (iii) the oracle's selection applied to the GPU's own fp32 scores reproduces kept_idx bit for bit (tie rule)
     (iv)  gathered K / V / position rows equal the source rows at the GPU's kept_idx, bit for bit
+    (v)   with res["sentinels"] (buffers of a GpuStep): nothing was written outside the valid regions -- rows at or
+          beyond r' of kept_idx / out_pos / out_k / out_v up to the request's capacity and score entries at or beyond
+          N_b still hold the initial fill
     """
     gm = cfg.group_mode if group_mode is None else group_mode
     G = cfg.n_kv_heads if gm == 0 else 1
@@ -122,6 +153,11 @@ def check_parity(cfg: wl.Config, st: dict, res: dict, ref_scores: np.ndarray, gr
     B = len(st["cache_len"])
     q_off, chunk_off, cache_off = st["q_off"], st["chunk_off"], st["cache_off"]
     summary = dict(units=0, band_keys=0, max_rel_err=0.0, swapped_units=0)
+    sentinels = bool(res.get("sentinels"))
+    if sentinels:
+        store_fill = np.uint32(SENTINEL_F32) if cfg.dtype == "f32" else np.uint16(SENTINEL_BF16)
+        store_bits = (lambda a: a.view(np.uint32)) if cfg.dtype == "f32" else (lambda a: a)
+        f32_bits = lambda a: np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
     for b in range(B):
         c = int(st["cache_len"][b])
         m = int(chunk_off[b + 1] - chunk_off[b])
@@ -129,9 +165,20 @@ def check_parity(cfg: wl.Config, st: dict, res: dict, ref_scores: np.ndarray, gr
         r = max(0, min(int(st["budget"][b]), N))
         assert int(res["out_len"][b]) == r, (b, res["out_len"][b], r)
         so, co, ho = int(cache_off[b] + chunk_off[b]), int(cache_off[b]), int(chunk_off[b])
+        cap = int(cache_off[b + 1] - cache_off[b])
         for l in range(L):
             for g in range(G):
                 summary["units"] += 1
+                if sentinels:
+                    assert np.all(f32_bits(res["scores"][l, g, so + N:so + cap + m]) == SENTINEL_F32), \
+                        f"scores written beyond the candidates b={b} l={l} g={g}"
+                    assert np.all(res["kept_idx"][l, g, co + r:co + cap] == SENTINEL_I32), "kept_idx beyond r'"
+                    assert np.all(res["out_pos"][l, g, co + r:co + cap] == SENTINEL_I32), "out_pos beyond r'"
+                    for kk in range(kvpg):
+                        for name_out in ("out_k", "out_v"):
+                            tail = store_bits(np.ascontiguousarray(res[name_out][l, g * kvpg + kk, co + r:co + cap]))
+                            assert np.all(tail == store_fill), f"{name_out} rows written beyond r' b={b} l={l}"
+
                 ref = ref_scores[l, g, so:so + N]
                 got = res["scores"][l, g, so:so + N].astype(np.float64)
                 if check_scores and N:

@@ -93,7 +93,7 @@ class _Fake:
         p = cls.base
         return fb.Batch(None, None, None, None, None,
                         fb.finch_batch(B, p, p + 256, p + 512, p + 768, p + 1024, total_q, total_chunk, total_cache,
-                                       max_q, max_cache, max_chunk, max_budget, 0))
+                                       max_q, max_cache, max_chunk, max_budget))
 
     @classmethod
     def tensor(cls, slot, tokens, d=64, heads=2, misalign=0, stride_tok=None):
@@ -134,6 +134,15 @@ def test_step_validation_paths(lib):
         # outputs may not alias inputs (parallel gather)
         assert _step(lib, ctx, good, ok=_Fake.tensor(1, 256)) == fb.FINCH_ERR_INVALID_ARG
         assert _step(lib, ctx, good, ov=_Fake.tensor(5, 256)) == fb.FINCH_ERR_INVALID_ARG
+        # ... nor overlap them partially: an output that starts inside cache_k's extent, or ends inside chunk_v's
+        assert _step(lib, ctx, good, ok=_Fake.tensor(1, 256, misalign=64 * 2 * 100)) == fb.FINCH_ERR_INVALID_ARG
+        assert _step(lib, ctx, good, ov=_Fake.tensor(4, 256, misalign=-64 * 2 * 200)) == fb.FINCH_ERR_INVALID_ARG
+        assert _step(lib, ctx, good, ov=_Fake.tensor(5, 256, misalign=16)) == fb.FINCH_ERR_INVALID_ARG
+        # K and V rows interleaved in one buffer (token stride 2 * head_dim, V shifted by one row) share no byte
+        inter = lambda slot, shift: _Fake.tensor(slot, 256, stride_tok=128, misalign=shift)
+        assert _step(lib, ctx, good, ok=inter(5, 0), ov=inter(5, 128)) == fb.FINCH_ERR_UNSUPPORTED
+        assert _step(lib, ctx, good, ok=inter(5, 0), ov=inter(5, 64)) == fb.FINCH_ERR_INVALID_ARG   # half a row
+        assert _step(lib, ctx, good, ck=inter(1, 0), ok=inter(1, 128)) == fb.FINCH_ERR_UNSUPPORTED
         # batch bounds against the context and against themselves
         assert _step(lib, ctx, _Fake.batch(B=5)) == fb.FINCH_ERR_INVALID_ARG
         assert _step(lib, ctx, _Fake.batch(max_q=65, total_q=128)) == fb.FINCH_ERR_INVALID_ARG

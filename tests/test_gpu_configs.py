@@ -58,8 +58,42 @@ def test_config_layers_full_width(name, layers_gpu, layers_checked):
     print(name, summary)
 
 
+@pytest.mark.parametrize("name,layers_checked", [
+    ("c2", [0, 7, 15, 31]),
+    ("c3", [0, 7, 15, 31]),
+    ("c5", [0, 7, 15, 31]),
+])
+def test_config_all_layers_in_the_benchmarked_geometry(name, layers_checked):
+    """The whole configuration -- all 32 layers in one step, i.e. the launch geometry bench.py times -- with the
+    oracle checking the first, the last and two inner layers.  Work is dealt to the persistent CTAs in contiguous
+    ranges of key tiles that do not line up with layers, so every checked layer holds units that straddle a range
+    boundary.  All layers are checked for what needs no oracle: the exact selection on the GPU's own scores, the
+    gathered rows, the planted keys and the untouched sentinels."""
+    cfg = wl.CONFIGS[name]
+    layers = list(range(cfg.n_layers))
+    st = wl.steady_state(cfg, layers)
+    g = GpuStep(cfg, st, len(layers))
+    try:
+        g.run()
+        assert g.status() == 0
+        res = g.results()
+    finally:
+        g.close()
+    sub = _slice_layers(st, layers_checked)
+    ref = oracle_scores(cfg, sub, threads=oracle.max_threads())
+    summary = check_parity(cfg, sub, _slice_results(res, layers_checked), ref)
+    # every layer: selection, gather and sentinels against the GPU's own scores (no oracle scores needed)
+    check_parity(cfg, st, res, res["scores"].astype(np.float64), check_scores=False)
+    planted = set(st["planted"][0].tolist())
+    r = int(st["budget"][0])
+    for l in layers:
+        for grp in range(cfg.n_groups):
+            assert planted <= set(res["kept_idx"][l, grp, :r].tolist()), "a planted key was dropped"
+    print(name, summary)
+
+
 def test_config4_ragged_batch_layer():
-    """The ragged batch at full shape for one layer; the oracle checks a sample of the requests."""
+    """The ragged batch at full shape for one layer; the oracle checks every request."""
     cfg = wl.CONFIGS["c4"]
     st = wl.steady_state(cfg, [3])
     g = GpuStep(cfg, st, 1)
@@ -70,8 +104,7 @@ def test_config4_ragged_batch_layer():
     finally:
         g.close()
     nqs = [r.n_q for r in cfg.requests]
-    sample = sorted({int(np.argmin(nqs)), int(np.argmax(nqs)), 0})   # shortest and longest prompt, and the first
-    for b in sample:
+    for b in range(cfg.batch):
         one = wl.scaled(cfg, requests=(cfg.requests[b],))
         sl = lambda off, a, ax: np.ascontiguousarray(np.take(a, np.arange(off[b], off[b + 1]), axis=ax))
         sub = dict(q=sl(st["q_off"], st["q"], 2), cache_k=sl(st["cache_off"], st["cache_k"], 2),
@@ -86,7 +119,7 @@ def test_config4_ragged_batch_layer():
         co, cap = int(st["cache_off"][b]), int(sub["cache_off"][1])
         rsub = dict(scores=res["scores"][:, :, so:so + n_cand], kept_idx=res["kept_idx"][:, :, co:co + cap],
                     out_len=res["out_len"][b:b + 1], out_pos=res["out_pos"][:, :, co:co + cap],
-                    out_k=res["out_k"][:, :, co:co + cap], out_v=res["out_v"][:, :, co:co + cap])
+                    out_k=res["out_k"][:, :, co:co + cap], out_v=res["out_v"][:, :, co:co + cap], sentinels=True)
         ref = oracle_scores(one, sub, threads=oracle.max_threads())
         check_parity(one, sub, rsub, ref)
 
@@ -194,6 +227,27 @@ def test_inconsistent_device_metadata_sets_the_status_word():
         g.run()
         assert g.status() & fb.FINCH_DEV_BAD_BATCH
         assert int(g.out_len.cpu()[0]) == 0
+        assert g.guards_intact()
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("which", ["q_off", "chunk_off", "cache_off"])
+def test_device_offsets_outside_the_packed_tensors_set_the_status_word(which):
+    """Offsets live in device memory and are only bounded by the host totals: a region that would start or end
+    outside its packed tensor is refused by every kernel (status word, unit skipped), never dereferenced."""
+    cfg = wl.scaled(wl.CONFIGS["c3"], n_layers=1, n_q_heads=4, n_kv_heads=2, head_dim=64,
+                    requests=(wl.Request(8, 9999, 40, 16),))
+    st = wl.steady_state(cfg, [0])
+    g = GpuStep(cfg, st, 1)
+    try:
+        getattr(g.batch, which).add_(5)      # same lengths, shifted past the end of the packed tensor
+        g.run()
+        assert g.status() & fb.FINCH_DEV_BAD_BATCH
+        assert int(g.out_len.cpu()[0]) == 0
+        assert g.guards_intact()
+        kept = g.kept_idx.cpu().numpy()
+        assert (kept == -1).all(), "a refused unit must leave its outputs alone"
     finally:
         g.close()
 

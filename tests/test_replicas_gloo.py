@@ -1,8 +1,10 @@
 """The N > 1 path of the benchmark on CPU: independent replicas, aggregated with gloo (world size 2).
 
 The step has no exchange between GPUs, so `bench.py --gpus N` runs N replicas; the only cross-rank logic is the
-aggregation of timings (slowest rank) and work (sum), which this test drives with two CPU processes.
+aggregation of timings (slowest rank) and work (sum), which this test drives with two CPU processes, and the
+launcher that starts the ranks when torchrun did not, which is run here with a stand-in rank on gloo.
 """
+import json
 import os
 import sys
 from pathlib import Path
@@ -38,3 +40,19 @@ def test_single_rank_needs_no_process_group():
     sys.path.insert(0, str(ROOT))
     import bench
     assert bench.aggregate_over_ranks(3.5, 100, 1, "gloo") == (3.5, 100)
+
+
+def test_launcher_starts_the_ranks_with_a_torchrun_style_environment(tmp_path):
+    """`bench.py --gpus 2` without torchrun: launch_replicas starts two processes that find each other."""
+    sys.path.insert(0, str(ROOT))
+    import bench
+    out = tmp_path / "line.json"
+    rc = bench.launch_replicas(2, [str(ROOT / "tests" / "replica_stub.py"), str(out)])
+    assert rc == 0
+    assert json.loads(out.read_text()) == {"n_gpus": 2, "ms": 3.0, "tokens": 3000}
+
+
+def test_launcher_reports_a_failed_rank(tmp_path):
+    sys.path.insert(0, str(ROOT))
+    import bench
+    assert bench.launch_replicas(2, ["-c", "import os, sys; sys.exit(3 if os.environ['RANK'] == '1' else 0)"]) == 3

@@ -65,7 +65,7 @@ def test_static_scratch_rejects_batches_beyond_its_size():
 
         def call(total_q):
             b = fb.finch_batch(1, base, base + 256, base + 512, base + 768, base + 1024, total_q, 512, 256,
-                               min(total_q, 4096), 256, 512, 256, 0)
+                               min(total_q, 4096), 256, 512, 256)
             t = lambda slot, tok, heads: fb.finch_tensor(base + 0x1000_0000 * slot, heads * tok * 64, tok * 64, 64)
             q, ck, hk = t(1, total_q, 32), t(2, 256, 8), t(3, 512, 8)
             return fb.load().finch_score_static(ctx, C.byref(q), C.byref(ck), C.byref(hk), C.byref(b),
