@@ -56,9 +56,11 @@ WsLayout ws_layout(const finch_ctx *ctx, const finch_batch *b) {
     const ModelView &mv = ctx->model;
     w.lse_off = 0;
     const size_t n_kv_scores = (size_t)mv.L * mv.Hkv * ((size_t)b->total_cache + b->total_chunk);
-    w.lse_bytes = align_up((size_t)mv.L * mv.Hq * (size_t)b->total_q * sizeof(float2) * (kScoreMaxSplits * 4 + 1) +
-                           (4 * n_kv_scores + 2) * sizeof(float) +  // row statistics, partial scores per KV head,
-                           ((size_t)b->batch + 1) * 8 + 4096);   // and the item plan of a multi-request batch
+    w.lse_bytes = (size_t)mv.L * mv.Hq * (size_t)b->total_q * sizeof(float2) * (kScoreMaxSplits * 4 + 1) +
+                  (4 * n_kv_scores + 2) * sizeof(float) +  // row statistics, partial scores per KV head,
+                  ((size_t)b->batch + 1) * 8 + 4096;       // and the item plan of a multi-request batch
+    const size_t fused = score_fused_scratch(*ctx, view_of(b)) * sizeof(float2);  // the one-kernel path's layout
+    w.lse_bytes = align_up(w.lse_bytes > fused ? w.lse_bytes : fused);
     w.scores_off = w.lse_off + w.lse_bytes;
     w.scores_bytes = align_up((size_t)mv.L * mv.G * ((size_t)b->total_cache + b->total_chunk) * sizeof(float));
     w.total = w.scores_off + w.scores_bytes;
@@ -144,7 +146,9 @@ cudaError_t run_score(const Ctx &ctx, const TensorView &q, const TensorView &cac
                       const BatchView &bv, float *scores, float2 *scratch, size_t scratch_capacity, float *row_lse,
                       cudaStream_t stream) {
     if (score_tc_supported(ctx)) {
-        const cudaError_t e =
+        cudaError_t e = launch_score_fused(ctx, q, cache_k, chunk_k, bv, scores, scratch, scratch_capacity, row_lse, stream);
+        if (e != cudaErrorNotSupported) return e;
+        e =
             launch_score_tc(ctx, q, cache_k, chunk_k, bv, scores, scratch, scratch_capacity, row_lse, stream);
         if (e != cudaErrorNotSupported) return e;
     }

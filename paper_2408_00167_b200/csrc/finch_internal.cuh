@@ -137,6 +137,13 @@ cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorVie
                             const BatchView &bv, float *scores, float2 *partial, size_t partial_capacity,
                             float *row_lse, cudaStream_t stream);
 
+// both sweeps in one persistent kernel (single-request batches without a row mask whose query tiles fit the shared
+// memory): score_fused_scratch gives the float2 entries of scratch it needs, 0 when it does not take the batch
+size_t score_fused_scratch(const Ctx &ctx, const BatchView &bv);
+cudaError_t launch_score_fused(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
+                               const BatchView &bv, float *scores, float2 *scratch, size_t scratch_capacity,
+                               float *row_lse, cudaStream_t stream);
+
 // scoring dispatch shared by finch_score, finch_score_static and finch_step; `scratch` holds scratch_capacity
 // float2 entries, at least one per prompt row (n_layers * n_q_heads * total_q)
 cudaError_t run_score(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
