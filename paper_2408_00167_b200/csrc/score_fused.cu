@@ -32,15 +32,18 @@ namespace {
 using namespace ptx;
 using namespace tc;
 
-constexpr int kFusedAuxBytes = 1024 + kStatsBytes;
+// barriers, then the row statistics: 4 groups x 2 buffers x `tiles` query tiles
+constexpr int fused_aux_bytes(int tiles) { return 1024 + kGroups * 2 * tiles * kRows * 8; }
 constexpr int kSoftmaxWarps = kGroups * 4;
+constexpr int kHelpers = 64;  // two helper warps: the exchange of row statistics and the sum over the groups
+constexpr int kFusedThreads = kTcThreads + kHelpers;
 constexpr int kMaxSegs = 8;  // ranges that may overlap one unit (bounds the partial-statistics array)
 
 struct FusedParams {
     ModelView mv;  // the scoring view: one unit per KV head
     BatchView bv;
     float2 *partial;     // [units][seg_max][kGroups][rows_u] (reference base-2 logit, sum exp2) per row and part
-    int *tickets;        // [units] softmax warps that have published their phase-A statistics of the unit
+    int *tickets;        // [units] ranges of the unit whose phase-A statistics are published
     float *row_lse;      // nullable
     float *unit_scores;  // [L][Hkv][cand]: the column sums of one KV head's query heads
     float *score_parts;  // [kGroups][L][Hkv][cand] per-group partial column sums
@@ -51,6 +54,7 @@ struct FusedParams {
     int stages;   // key-tile ring depth
     int q_tiles;  // resident query tiles (= query tiles of a unit, at most kQTiles)
     int delay;    // 0: phase B of a window right after its phase A; 1: one window later
+    int stats_tiles;  // room, in query tiles, of a softmax group's statistics buffer (3 when a unit can have 3 tiles)
 };
 
 __device__ __forceinline__ int ld_acquire_gpu(const int *p) {
@@ -67,6 +71,24 @@ __device__ __forceinline__ bool ticket_wait(const int *ticket, int target, volat
         if (ld_acquire_gpu(ticket) >= target) return true;
         if (*abort_flag) return false;
         __nanosleep(it < 256 ? 40 : 400);
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+// A counter in shared memory that some warps bump (after their writes) and another polls (before its reads).
+__device__ __forceinline__ void count_arrive(int *counter) {
+    __threadfence_block();
+    atomicAdd_block(counter, 1);
+}
+__device__ __forceinline__ bool count_wait(int *counter, int target, volatile int *abort_flag) {
+    for (uint32_t it = 0; it < kTicketSpins; ++it) {
+        if (*(volatile int *)counter >= target) {
+            __threadfence_block();
+            return true;
+        }
+        if (*abort_flag) return false;
+        __nanosleep(64);
     }
     *abort_flag = 1;
     return false;
@@ -101,7 +123,7 @@ __device__ __forceinline__ bool next_seg(const Geo &g, int W, int rho, int &x, i
 }
 
 template <int D>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kFusedThreads, 1)
 score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap cache_map,
                    const __grid_constant__ CUtensorMap chunk_map, FusedParams p) {
     constexpr int kSlabs = D / 64;
@@ -117,11 +139,14 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     uint64_t *empty = full + kMaxStages;
     uint64_t *acc_full = empty + kMaxStages;
     uint64_t *acc_empty = acc_full + kAccBufs;
-    uint64_t *stats_ready = acc_empty + kAccBufs;  // all softmax warps have staged their share of the statistics
-    uint64_t *seg_done = stats_ready + 1;          // all softmax warps have written their partial column sums
-    uint32_t *tmem_slot = (uint32_t *)(seg_done + 1);
+    uint64_t *grp_ready = acc_empty + kAccBufs;  // [kGroups] the group's warps have staged their row statistics
+    uint32_t *tmem_slot = (uint32_t *)(grp_ready + kGroups);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
-    float2 *stats_sm = (float2 *)(aux + 1024);  // [2][q_tiles * 128] row statistics of phase B, double-buffered
+    // Softmax warps -> helpers: plain counters (one count per warp and segment), not barrier phases, so that a helper
+    // that falls behind by more than one segment still reads the right answer.
+    int *a_count = (int *)(tmem_slot + 2);  // softmax warps that have written a phase-A segment's statistics
+    int *b_count = a_count + 1;             // softmax warps that are through a phase-B segment
+    float2 *stats_sm = (float2 *)(aux + 1024);  // [kGroups][2][stats_tiles * 128] row statistics of phase B
 
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
@@ -136,8 +161,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             mbar_init(&acc_full[b], 1);
             mbar_init(&acc_empty[b], 4);  // one arrival per softmax warp of the owning group
         }
-        mbar_init(stats_ready, kSoftmaxWarps);
-        mbar_init(seg_done, kSoftmaxWarps);
+        for (int b = 0; b < kGroups; ++b) mbar_init(&grp_ready[b], 4);
+        *a_count = 0;
+        *b_count = 0;
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -276,8 +302,10 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 }
             })
         }
-    } else {
+    } else if (warp < 2 + kSoftmaxWarps) {
         // =================================================================== softmax warps (one TMEM lane per thread)
+        // They only compute: what has to be exchanged with other CTAs, merged or summed across the groups is the
+        // helper warps' business, and every barrier they wait on is normally complete when they get there.
         const int quarter = warp & 3;            // tcgen05.ld reaches lanes 32 * (warp % 4) ..
         const int sw = warp - 2;                 // softmax warp 0..15
         const int grp = sw >> 2;                 // softmax group = the accumulator buffer it owns
@@ -286,10 +314,12 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const float scale2 = mv.scale * kLog2e;
         const int64_t cand = (int64_t)bv.total_cache + bv.total_chunk;
         const int64_t units = (int64_t)mv.L * mv.G;
-        int A = 0, mine = 0, epoch = 0, segs_b = 0;
+        const int gcd4 = (g.n_qt & 3) == 0 ? 4 : ((g.n_qt & 1) == 0 ? 2 : 1);  // gcd(query tiles, softmax groups)
+        // query tiles whose statistics this group stages: its own one when the tiles divide the groups, else all
+        const int st_tiles = g.n_qt > 0 && 4 % g.n_qt == 0 ? 1 : g.n_qt;
+        int A = 0, mine = 0, segs_b = 0, epoch = 0;
         bool ok = true;
         FINCH_FOR_EACH_SEGMENT({
-            float2 *part_stats = p.partial + ((int64_t)sg.unit * p.seg_max) * kGroups * p.rows_u;
             if (ph == 0) {
                 // ---------------------------------------------------------------- phase A: row statistics
                 float m_raw[kQTiles], z[kQTiles];
@@ -330,8 +360,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     }
                 }
                 if (!ok) break;
-                // publish: every group reports every resident row, (-inf, 0) where it saw no accumulator
-                float2 *dst = part_stats + ((int64_t)sg.slot * kGroups + grp) * p.rows_u;
+                // hand the statistics to the helper warps: every group reports every resident row, (-inf, 0) where
+                // it saw no accumulator
+                float2 *dst = p.partial + (((int64_t)sg.unit * p.seg_max + sg.slot) * kGroups + grp) * p.rows_u;
 #pragma unroll
                 for (int qb = 0; qb < kQTiles; ++qb) {
                     if (qb >= g.n_qt) continue;
@@ -339,59 +370,64 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     const int r = my_row % kSub;
                     if (r < sb.valid) dst[sb.hh * bv.max_q + sb.p0 + r] = make_float2(m_raw[qb] * scale2, z[qb]);
                 }
-                __threadfence();
                 __syncwarp();
-                if (lane == 0) atomicAdd(&p.tickets[sg.unit], 1);
+                if (lane == 0) count_arrive(a_count);
             } else {
                 // ---------------------------------------------------------------- phase B: column sums
-                // all ranges of the unit have published once every softmax warp of each has bumped the ticket
+                // all ranges of the unit have published their statistics once the ticket says so (with delay = 1
+                // that was a window ago)
                 int published = 1;
-                if (lane == 0) published = ticket_wait(&p.tickets[sg.unit], kSoftmaxWarps * sg.n_seg, abort_flag);
+                if (lane == 0) published = ticket_wait(&p.tickets[sg.unit], sg.n_seg, abort_flag);
                 if (!__shfl_sync(0xffffffffu, published, 0)) {
                     ok = false;
                     break;
                 }
-                // Merge the parts of the resident rows (fixed order: ranges, then groups) and stage (-R, w): every
-                // softmax warp its share, into one of two buffers; a warp that has passed the barrier of epoch e
-                // has seen all warps finish epoch e - 1, so the buffer of epoch e + 1 (= that of e - 1) is free.
+                // Each group merges and stages what its own accumulators will need -- one query tile when the tiles
+                // of a unit divide the four groups (its number is then fixed: accumulator A goes to group A % 4),
+                // all of them otherwise -- one row per thread, parts in a fixed order (ranges, then groups).  Only the
+                // group's four warps meet at the barrier, and they move in step anyway.  Two buffers: a warp past the
+                // barrier of epoch e has seen its group finish epoch e - 1, so the buffer of e + 1 is free.
+                float2 *sm_grp = stats_sm + ((grp * 2 + (epoch & 1)) * p.stats_tiles) * kRows;
                 {
-                    float2 *stage_to = stats_sm + (epoch & 1) * kQTiles * kRows;
-                    const int n_parts = sg.n_seg * kGroups;
-                    for (int idx = sw * 32 + lane; idx < g.n_qt * kRows; idx += kSoftmaxWarps * 32) {
-                        const int r = idx % kRows;
-                        const SubBlock sb = sub_block(2 * (idx / kRows) + r / kSub, g.sbq, g.n_sb, u.n_q);
+                    const float2 *part_stats = p.partial + ((int64_t)sg.unit * p.seg_max) * kGroups * p.rows_u;
+                    const int r = (sw & 3) * 32 + lane;  // this thread's row of the tile
+                    for (int qs = 0; qs < st_tiles; ++qs) {
+                        const int qb = st_tiles == 1 ? grp % g.n_qt : qs;
+                        const SubBlock sb = sub_block(2 * qb + r / kSub, g.sbq, g.n_sb, u.n_q);
                         float2 out = make_float2(0.f, 0.f);
-                        if (r % kSub < sb.valid) {
+                        if (qb < g.n_qt && r % kSub < sb.valid) {
                             const int pr = sb.p0 + r % kSub;
                             const float2 *src = part_stats + sb.hh * bv.max_q + pr;
                             float M = -INFINITY, Z = 0.f;
-#pragma unroll 1
-                            for (int i0 = 0; i0 < n_parts; i0 += 8) {
-                                float2 part[8];
+                            // group g' has met tile qb only if g' - qb is a multiple of gcd(tiles, groups)
+#pragma unroll 2
+                            for (int sgi = 0; sgi < sg.n_seg; ++sgi) {
+                                float2 part[kGroups];
 #pragma unroll
-                                for (int i = 0; i < 8; ++i)
-                                    part[i] = i0 + i < n_parts ? __ldcg(src + (int64_t)(i0 + i) * p.rows_u)
-                                                               : make_float2(0.f, 0.f);
+                                for (int k = 0; k < kGroups; ++k)
+                                    part[k] = ((k - qb) & (gcd4 - 1)) == 0
+                                                  ? __ldcg(src + ((int64_t)sgi * kGroups + k) * p.rows_u)
+                                                  : make_float2(0.f, 0.f);
 #pragma unroll
-                                for (int i = 0; i < 8; ++i) merge_part(part[i], M, Z);
+                                for (int k = 0; k < kGroups; ++k) merge_part(part[k], M, Z);
                             }
                             const int64_t row = ((int64_t)u.l * mv.Hq + u.G * mv.hpg + sb.hh) * bv.total_q + u.q0 + pr;
                             if (bv.self_lse) merge_self_term(bv.self_lse[row], M, Z);
                             float lse_nat;
                             out = merged_pair(M, Z, lse_nat);
-                            if (p.row_lse && sg.slot == 0) p.row_lse[row] = lse_nat;  // once per unit
+                            // once per unit: its first range, and the one group whose number is the tile's
+                            if (p.row_lse && sg.slot == 0 && (st_tiles == 1 ? grp == qb : grp == 0)) p.row_lse[row] = lse_nat;
                         }
                         // rows 2k and 2k+1 share one float4: (-ref_2k, -ref_2k+1, w_2k, w_2k+1)
-                        float *smf = (float *)stage_to + (idx >> 1) * 4 + (idx & 1);
+                        float *smf = (float *)(sm_grp + qs * kRows) + (r >> 1) * 4 + (r & 1);
                         smf[0] = out.x;
                         smf[2] = out.y;
                     }
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(stats_ready);
-                    if (!__all_sync(0xffffffffu, mbar_wait(stats_ready, epoch & 1, abort_flag))) { ok = false; break; }
+                    if (lane == 0) mbar_arrive(&grp_ready[grp]);
+                    if (!__all_sync(0xffffffffu, mbar_wait(&grp_ready[grp], epoch & 1, abort_flag))) { ok = false; break; }
                     ++epoch;
                 }
-                const float2 *sm = stats_sm + ((epoch - 1) & 1) * kQTiles * kRows;
                 float *part = p.score_parts + ((int64_t)grp * units + sg.unit) * cand + u.cache0 + u.chunk0;
                 for (int t = sg.t0; t < sg.t1 && ok; ++t) {
                     const KeyTile kt = key_tile(u, t);
@@ -404,7 +440,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                         tc_fence_after();
                         const int v0 = sub_block(2 * qb, g.sbq, g.n_sb, u.n_q).valid;
                         const int v1 = sub_block(2 * qb + 1, g.sbq, g.n_sb, u.n_q).valid;
-                        colsum_accumulate<false>(t_acc, v0, v1, scale2, sm + qb * kRows, c0, c1, nullptr, 0);
+                        colsum_accumulate<false>(t_acc, v0, v1, scale2, sm_grp + (st_tiles == 1 ? 0 : qb) * kRows, c0, c1, nullptr, 0);
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&acc_empty[grp]);
@@ -412,22 +448,50 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     if (ok && my_row < kt.valid) part[kt.j0 + my_row] = c0 + c1;  // 0 if the group had no accumulator
                 }
                 if (!ok) break;
-                // the four groups' partial sums of this segment's keys, added in group order
+                // this warp's partial sums are written: the helper warps add the four groups' sums
                 __syncwarp();
-                if (lane == 0) mbar_arrive(seg_done);
-                if (!__all_sync(0xffffffffu, mbar_wait(seg_done, segs_b & 1, abort_flag))) { ok = false; break; }
+                if (lane == 0) count_arrive(b_count);
                 ++segs_b;
-                {
-                    const KeyTile first = key_tile(u, sg.t0), last = key_tile(u, sg.t1 - 1);
-                    const int j_end = last.j0 + last.valid;
-                    const float *parts0 = p.score_parts + (int64_t)sg.unit * cand + u.cache0 + u.chunk0;
-                    float *out = p.unit_scores + (int64_t)sg.unit * cand + u.cache0 + u.chunk0;
-                    for (int j = first.j0 + sw * 32 + lane; j < j_end; j += kSoftmaxWarps * 32) {
-                        float s = 0.f;
+            }
+        })
+    } else {
+        // =================================================================== helper warps
+        // What has to leave the CTA or cross the groups, off the softmax warps' path; they walk the same schedule
+        // as everyone.  After a phase-A segment, once the softmax warps have written their statistics, one thread
+        // makes them visible to the GPU and bumps the unit's ticket (neighbouring CTAs wait for it).  After a
+        // phase-B segment the 64 threads add the four groups' partial column sums, in group order.
+        const int tid = threadIdx.x - (2 + kSoftmaxWarps) * 32;
+        const int64_t cand = (int64_t)bv.total_cache + bv.total_chunk;
+        const int64_t units = (int64_t)mv.L * mv.G;
+        int segs_a = 0, segs_b = 0;
+        bool ok = true;
+        auto warp_agree = [&](bool good) -> bool { return __all_sync(0xffffffffu, good); };
+        FINCH_FOR_EACH_SEGMENT({
+            if (ph == 0) {
+                ++segs_a;
+                if (tid >= 32) continue;  // the first helper warp's business
+                if (!warp_agree(lane != 0 || count_wait(a_count, kSoftmaxWarps * segs_a, abort_flag))) { ok = false; break; }
+                if (lane == 0) {
+                    __threadfence();  // cumulative: covers the softmax warps' stores this thread has synchronised with
+                    atomicAdd(&p.tickets[sg.unit], 1);
+                }
+            } else {
+                ++segs_b;
+                if (!warp_agree(lane != 0 || count_wait(b_count, kSoftmaxWarps * segs_b, abort_flag))) { ok = false; break; }
+                const KeyTile first = key_tile(u, sg.t0), last = key_tile(u, sg.t1 - 1);
+                const int j_end = last.j0 + last.valid;
+                const float *parts0 = p.score_parts + (int64_t)sg.unit * cand + u.cache0 + u.chunk0;
+                float *out = p.unit_scores + (int64_t)sg.unit * cand + u.cache0 + u.chunk0;
+                for (int j = first.j0 + tid; j < j_end; j += kHelpers * 4) {  // four keys in flight per thread
+                    float v[4][kGroups];
 #pragma unroll
-                        for (int k = 0; k < kGroups; ++k) s += __ldcg(parts0 + (int64_t)k * units * cand + j);
-                        out[j] = s;
-                    }
+                    for (int i = 0; i < 4; ++i)
+#pragma unroll
+                        for (int k = 0; k < kGroups; ++k)
+                            v[i][k] = j + kHelpers * i < j_end ? parts0[(int64_t)k * units * cand + j + kHelpers * i] : 0.f;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        if (j + kHelpers * i < j_end) out[j + kHelpers * i] = ((v[i][0] + v[i][1]) + v[i][2]) + v[i][3];
                 }
             }
         })
@@ -503,9 +567,10 @@ cudaError_t launch_fused_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensor
     constexpr int kTileBytes = (D / 64) * kSlabBytes;
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
-    p.stages = min(kMaxStages, (kSmemLimit - 1024 - kFusedAuxBytes - p.q_tiles * kTileBytes) / kTileBytes);
+    const int aux = fused_aux_bytes(p.stats_tiles);
+    p.stages = min(kMaxStages, (kSmemLimit - 1024 - aux - p.q_tiles * kTileBytes) / kTileBytes);
     if (p.stages < 2) return cudaErrorNotSupported;
-    const int smem = 1024 + (p.q_tiles + p.stages) * kTileBytes + kFusedAuxBytes;
+    const int smem = 1024 + (p.q_tiles + p.stages) * kTileBytes + aux;
     cudaError_t e = cudaFuncSetAttribute(score_fused_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     const int units = mv.L * mv.G;
@@ -513,7 +578,7 @@ cudaError_t launch_fused_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensor
     if (e != cudaSuccess) return e;
     const int sms = ctx.sm_count > 0 ? ctx.sm_count : 148;
     dim3 grid(n_ranges < sms ? n_ranges : sms);  // persistent and resident at once: phase B waits for neighbours
-    e = launch_chained(score_fused_kernel<D>, grid, dim3(kTcThreads), smem, stream, qm, cm, hm, p);
+    e = launch_chained(score_fused_kernel<D>, grid, dim3(kFusedThreads), smem, stream, qm, cm, hm, p);
     ctx.launches += 2;
     if (e != cudaSuccess || heads_per_group == 1) return e;
     dim3 sgrid((bv.max_cache + bv.max_chunk + 255) / 256, mv.L * out_groups);
@@ -576,6 +641,7 @@ cudaError_t launch_score_fused(const Ctx &ctx, const TensorView &q, const Tensor
     p.rows_u = mv.g * bv.max_q;
     p.q_tiles = (mv.g * ((bv.max_q + kSub - 1) / kSub) + 1) / 2;
     p.delay = 1;
+    p.stats_tiles = p.q_tiles >= 3 ? 3 : 1;  // a unit with three tiles (4 % 3 != 0) stages all of them per group
     if (const char *e = getenv("FINCH_FUSED_W")) p.W = max(1, min(tiles, atoi(e)));  // TEMP tuning knobs
     if (const char *e = getenv("FINCH_FUSED_DELAY")) p.delay = atoi(e) ? 1 : 0;
     if ((tiles + p.W - 1) / p.W + 1 > kMaxSegs) return cudaErrorNotSupported;
