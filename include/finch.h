@@ -168,17 +168,24 @@ finch_status finch_score(finch_ctx *ctx, const finch_tensor *prompt_q, const fin
                          const finch_tensor *chunk_k, const finch_batch *batch, float *scores, float *row_lse,
                          void *ws, size_t ws_bytes, void *cuda_stream);
 
-/* Same computation and outputs as finch_score, for callers that cannot allocate device memory.  (The paper has no
+/* The same scores and row_lse as finch_score, for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is an integration aid.)  Some hosts of this library may not call cudaMalloc at all -- a plugin
  * inside a serving process whose memory pool owns the whole device, or a step that must stay clear of the driver's
- * allocator for latency reasons -- and so cannot supply finch_score's workspace.  Here the per-row softmax
- * statistics that finch_score keeps in that workspace live in a fixed array inside the library image instead
- * (8 MiB of device memory on every GPU that loads the library, held until the process exits).  The call itself
- * allocates and frees nothing.
+ * allocator for latency reasons -- and so cannot supply finch_score's workspace.  Here everything finch_score
+ * keeps in that workspace lives in a fixed array inside the library image instead (8 MiB of device memory on every
+ * GPU that loads the library, held until the process exits).  The call itself allocates and frees nothing.
  *  - Limit: n_layers * n_q_heads * total_q must not exceed finch_score_static_max_rows() (2^20 rows); a larger
  *    batch is rejected with FINCH_ERR_WORKSPACE_TOO_SMALL and nothing is enqueued -- use finch_score then.
- *  - The first call on each device looks up the array's device address; the context's device must be the current
- *    device (FINCH_ERR_INVALID_ARG otherwise).  Make that first call before starting any stream capture.
+ *  - Which kernels run: the tensor-core kernels need more of the array than one entry per prompt row (in 8-byte
+ *    entries, for a single request: 32 per prompt row plus 2 per layer, KV head and candidate; for a batch of
+ *    requests: 5 per prompt row plus the same 2 per candidate).  A batch within the row limit whose need
+ *    exceeds the array's 2^20 entries -- a whole 32-layer step of 4096 candidates does -- runs on the warp-level
+ *    kernels instead: the same result within the score tolerance, many times slower.  finch_score_static_path
+ *    tells which it will be.  Because the kernels (or their key ranges) can differ from finch_score's, the two
+ *    calls agree within the score tolerance, max(1e-3 relative, 1e-5 absolute), not bit for bit.
+ *  - The first call on each device looks up the array's device address.  Make that first call before starting any
+ *    stream capture.  On EVERY call the context's device must be the current device (FINCH_ERR_INVALID_ARG
+ *    otherwise): the address belongs to that GPU.
  *  - Every call on a device shares the one array, which keeps the previous call's contents.  Nothing in it has
  *    to start at zero: each call overwrites every entry it later reads.  Two calls whose kernels overlap on the
  *    GPU (different streams, or different contexts on one device) race on it: serialise them. */
@@ -188,6 +195,12 @@ finch_status finch_score_static(finch_ctx *ctx, const finch_tensor *prompt_q, co
 
 /* The row limit of finch_score_static. */
 size_t finch_score_static_max_rows(void);
+
+/* Host arithmetic, nothing is enqueued: *tensor_cores = 1 when finch_score_static would run this batch on the
+ * tensor-core kernels (bf16, head_dim 64 or 128, and the batch's scratch fits the built-in array), 0 when it would
+ * take the warp-level kernels.  (The paper has no counterpart.)  A batch whose tensors the TMA unit cannot describe
+ * (an outer stride of 2^40 bytes or more) takes the warp-level kernels regardless. */
+finch_status finch_score_static_path(const finch_ctx *ctx, const finch_batch *batch, int32_t *tensor_cores);
 
 /* Top-r selection (Method, bullet "Selection of top r position": t = top-r(A^agg, r)).  For every layer, group and
  * request keeps r' = min(budget[b], N_b) candidates with the largest scores; among equal scores the lower

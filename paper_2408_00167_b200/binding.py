@@ -32,7 +32,8 @@ FINCH_GROUP_PER_KV_HEAD, FINCH_GROUP_PER_LAYER = 0, 1
 FINCH_DEV_BAD_BATCH, FINCH_DEV_TIMEOUT, FINCH_DEV_BAD_INDEX = 1, 2, 4
 
 EXPORTS = ("finch_ctx_create", "finch_ctx_destroy", "finch_workspace_bytes", "finch_score", "finch_select",
-           "finch_compact", "finch_step", "finch_device_status", "finch_launch_count", "finch_status_string", "finch_score_static", "finch_score_static_max_rows", "finch_step_host")
+           "finch_compact", "finch_step", "finch_device_status", "finch_launch_count", "finch_status_string", "finch_score_static", "finch_score_static_max_rows", "finch_score_static_path",
+           "finch_step_host")
 
 
 class finch_config(C.Structure):
@@ -237,6 +238,13 @@ def finch_score_static(ctx, prompt_q, cache_k, chunk_k, batch: Batch, scores, ro
 
 def finch_score_static_max_rows() -> int:
     return int(load().finch_score_static_max_rows())
+
+
+def finch_score_static_path(ctx, batch: Batch) -> bool:
+    """True when finch_score_static would run this batch on the tensor-core kernels, False: warp-level kernels."""
+    out = C.c_int32()
+    _check(load().finch_score_static_path(ctx, C.byref(batch.c), C.byref(out)), "finch_score_static_path")
+    return bool(out.value)
 
 
 def finch_step_host(ctx, host_prompt_q, host_chunk_k, host_chunk_v, host_chunk_pos, stage_q, stage_chunk_k,

@@ -467,10 +467,10 @@ finch_status finch_device_status(finch_ctx *ctx, void *cuda_stream, int32_t *out
 // ---------------------------------------------------------------------------------------------------------------
 // finch_score_static: scoring for callers that cannot allocate device memory.
 //
-// finch_score keeps one (row maximum, 1 / row sum) pair per prompt row between its two kernels, in a workspace the
-// caller allocates.  Code that runs where cudaMalloc is off limits -- a plugin inside a serving process that owns
+// finch_score keeps its intermediate results -- per-row softmax statistics, per-group partial column sums, a few
+// counters -- in a workspace the caller allocates.  Code that runs where cudaMalloc is off limits -- a plugin inside a serving process that owns
 // all device memory and hands none out, a callback that may not block on the allocator, a latency-critical loop
-// that must not touch the driver's heap -- has no such workspace to give.  For those callers the pairs live in the
+// that must not touch the driver's heap -- has no such workspace to give.  For those callers the scratch is the
 // fixed array below, which is part of the library image: every GPU that loads libfinch holds it until the process
 // exits.
 namespace {
@@ -522,3 +522,17 @@ extern "C" finch_status finch_score_static(finch_ctx *ctx, const finch_tensor *p
 }
 
 extern "C" size_t finch_score_static_max_rows(void) { return kStaticRows; }
+
+// Which kernels finch_score_static runs for a batch: the tensor-core kernels keep more than one entry per prompt row
+// in the scratch (statistics per key range and softmax group, partial column sums per candidate), so a batch can
+// fit the array's row limit and still be too large for them; it then takes the warp-level kernels.
+extern "C" finch_status finch_score_static_path(const finch_ctx *ctx, const finch_batch *batch, int32_t *tensor_cores) {
+    if (!tensor_cores) return FINCH_ERR_INVALID_ARG;
+    finch_status s = check_batch(ctx, batch);
+    if (s) return s;
+    const BatchView bv = view_of(batch);
+    const size_t fused = score_fused_scratch(*ctx, bv);
+    *tensor_cores = score_tc_supported(*ctx) &&
+                    ((fused > 0 && fused <= kStaticRows) || score_tc_scratch_min(*ctx, bv) <= kStaticRows);
+    return FINCH_OK;
+}

@@ -133,6 +133,7 @@ cudaError_t launch_score_simt(const Ctx &ctx, const TensorView &q, const TensorV
 // holds one float2 per prompt row and key split; up to kScoreMaxSplits splits are used when it is large enough.
 constexpr int kScoreMaxSplits = 8;
 bool score_tc_supported(const Ctx &ctx);
+size_t score_tc_scratch_min(const Ctx &ctx, const BatchView &bv);  // least scratch (float2) of the two-launch path
 cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
                             const BatchView &bv, float *scores, float2 *partial, size_t partial_capacity,
                             float *row_lse, cudaStream_t stream);

@@ -22,8 +22,6 @@
 //
 // Roles and barriers are those of the two-launch kernels (score_tc.cu): TMA producer lane, MMA issuer lane, four
 // softmax groups of four warps, accumulators dealt round-robin to the groups, every wait bounded.
-#include <stdlib.h>
-
 #include "score_tc_common.cuh"
 
 namespace finch {
@@ -642,8 +640,6 @@ cudaError_t launch_score_fused(const Ctx &ctx, const TensorView &q, const Tensor
     p.q_tiles = (mv.g * ((bv.max_q + kSub - 1) / kSub) + 1) / 2;
     p.delay = 1;
     p.stats_tiles = p.q_tiles >= 3 ? 3 : 1;  // a unit with three tiles (4 % 3 != 0) stages all of them per group
-    if (const char *e = getenv("FINCH_FUSED_W")) p.W = max(1, min(tiles, atoi(e)));  // TEMP tuning knobs
-    if (const char *e = getenv("FINCH_FUSED_DELAY")) p.delay = atoi(e) ? 1 : 0;
     if ((tiles + p.W - 1) / p.W + 1 > kMaxSegs) return cudaErrorNotSupported;
     const int n_ranges = (int)(((long long)units * tiles + p.W - 1) / p.W);
     return mv.d == 64 ? launch_fused_d<64>(ctx, qm, cm, hm, p, n_ranges, ctx.model.G, ctx.model.kvpg, scores, stream)

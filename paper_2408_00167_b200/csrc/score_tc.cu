@@ -663,6 +663,14 @@ bool score_tc_supported(const Ctx &ctx) {
     return ctx.cfg.dtype == FINCH_BF16 && (ctx.model.d == 64 || ctx.model.d == 128);
 }
 
+// The least scratch (float2 entries) the two-launch tensor-core path needs for this batch: one key split.
+size_t score_tc_scratch_min(const Ctx &ctx, const BatchView &bv) {
+    const ModelView &mv = ctx.model;
+    const size_t rows = (size_t)mv.L * mv.Hq * (size_t)bv.total_q;
+    const size_t cand = (size_t)mv.L * mv.Hkv * ((size_t)bv.total_cache + bv.total_chunk);
+    return rows * (kGroups + 1) + (kGroups * cand + 1) / 2 + (size_t)bv.batch + 1 + kPlanBoundsInts / 2;
+}
+
 // `partial` holds partial_capacity float2 entries; the key-split count is limited so that one entry per prompt
 // row, split and softmax group, one merged entry per row and the per-group partial scores fit.  Returns cudaErrorNotSupported (and launches nothing) when the tensors cannot be described
 // to the TMA unit; the caller then uses the warp-level path for every request.

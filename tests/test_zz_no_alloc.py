@@ -4,7 +4,10 @@ Some users of the library run where cudaMalloc is not an option (a plugin inside
 the device, a step that must not touch the driver's allocator).  They call finch_score_static, whose scratch is a
 fixed array inside the library instead of a caller-supplied workspace.  These tests check that it returns what
 finch_score returns, call after call, although every call reuses the same array, and that it refuses batches that
-do not fit the array.  The file is named to be collected last.
+do not fit the array.  The array is 8 MiB; the tensor-core kernels need more of it than one entry per prompt row, so a
+batch with few prompt rows but very many candidates stays within the row limit and still has to run on the warp-level
+kernels: that case is driven on purpose, and both kinds of batch are compared with the fp64 oracle, not only with
+finch_score.  The file is named to be collected last.
 """
 import ctypes as C
 
@@ -14,7 +17,7 @@ import pytest
 from paper_2408_00167_b200 import binding as fb
 from paper_2408_00167_b200 import build as fbuild
 from paper_2408_00167_b200 import workloads as wl
-from parity_harness import ABS_TOL, REL_TOL, GpuStep
+from parity_harness import ABS_TOL, REL_TOL, GpuStep, oracle_scores
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -52,6 +55,33 @@ def test_static_scratch_matches_workspace_version_on_consecutive_calls():
                 np.testing.assert_allclose(got_lse.cpu().numpy(), want_lse.cpu().numpy(), rtol=1e-5, atol=1e-5)
         finally:
             g.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("reqs,tensor_cores", [
+    ([(40, 10 ** 7, 700, 300)], True),          # a small batch: the tensor-core kernels fit the array
+    ([(33, 10 ** 7, 140_000, 200)], False),     # 4 units x 140 200 candidates of partial sums do not: warp-level kernels
+])
+def test_static_scratch_on_both_kernel_paths_against_the_oracle(reqs, tensor_cores):
+    import torch
+    cfg, st = _case(reqs, 1)
+    g = GpuStep(cfg, st, 2)
+    try:
+        assert fb.finch_score_static_path(g.ctx, g.batch) is tensor_cores
+        ref = oracle_scores(cfg, st, threads=8)
+        fb.finch_score(g.ctx, g.q, g.cache_k, g.chunk_k, g.batch, g.scores, g.row_lse, g.ws)   # always tensor cores
+        want = g.scores.clone()
+        for _ in range(2):
+            got = torch.full_like(g.scores, float("nan"))
+            fb.finch_score_static(g.ctx, g.q, g.cache_k, g.chunk_k, g.batch, got, None)
+            assert g.status() == 0
+            for name, x in (("static", got), ("workspace", want)):
+                x = x.cpu().numpy().astype(np.float64)
+                assert not np.isnan(x).any()
+                bad = np.abs(x - ref) > np.maximum(REL_TOL * np.abs(ref), ABS_TOL)
+                assert not bad.any(), f"{name}: {int(bad.sum())} scores outside the tolerance"
+    finally:
+        g.close()
 
 
 def test_static_scratch_rejects_batches_beyond_its_size():
