@@ -285,9 +285,9 @@ def run_ours(args, cfg: wl.Config):
     assert fb.finch_device_status(ctx) == 0
     launches0 = fb.finch_launch_count(ctx)
     t_begin = time.time()
-    block_ms = [timed(step, args.steps) for _ in range(BLOCKS)]
+    block_ms = [timed(step, args.steps) for _ in range(max(1, args.blocks))]
     t_end = time.time()
-    launches = (fb.finch_launch_count(ctx) - launches0) // BLOCKS       # per block of --steps steps
+    launches = (fb.finch_launch_count(ctx) - launches0) // max(1, args.blocks)   # per block of --steps steps
     assert fb.finch_device_status(ctx) == 0
     ms_local = statistics.median(block_ms)
     ms, tokens = aggregate_over_ranks(ms_local, counts["tokens"], world, "nccl")
@@ -330,7 +330,7 @@ def run_ours(args, cfg: wl.Config):
     line = {
         "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-        "timing": {"blocks": BLOCKS, "steps_per_block": args.steps, "statistic": "median block / steps",
+        "timing": {"blocks": max(1, args.blocks), "steps_per_block": args.steps, "statistic": "median block / steps",
                    "block_ms_min": min(block_ms), "block_ms_max": max(block_ms),
                    # time x clock: comparable between runs that saw different SM clocks
                    "kclk_per_step": ms_local * clocks["sm_mhz"] if clocks.get("sm_mhz") else None},
@@ -440,6 +440,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (small profiling runs)")
+    ap.add_argument("--blocks", type=int, default=BLOCKS, help="timed blocks of --steps steps (fewer for profiling runs)")
     ap.add_argument("--document", default="", choices=["", "fixed", "paper"],
                     help="also time the whole chunk loop with this budget schedule (adds a document_loop object)")
     ap.add_argument("--group-mode", type=int, default=-1, choices=[-1, 0, 1],

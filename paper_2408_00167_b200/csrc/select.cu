@@ -9,8 +9,8 @@
 namespace finch {
 namespace {
 
-constexpr int kSelThreads = 1024;
-constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kSelThreadsWide = 1024;  // units of more than 1024 candidates: two CTAs per SM
+constexpr int kSelThreadsSmall = 256;  // short units: eight CTAs per SM, so that many small units run in one wave
 
 // Order-preserving key: larger score <=> larger key.  -0 is folded into +0; NaN gets key 0, below every number.
 __device__ __forceinline__ uint32_t order_key(float s) {
@@ -20,9 +20,12 @@ __device__ __forceinline__ uint32_t order_key(float s) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// two CTAs per SM (32 registers per thread): c3's 256 units then run in one wave
-__global__ void __launch_bounds__(kSelThreads, 2)
+// 32 registers per thread, so 2048 threads per SM whatever the CTA size: two CTAs of 1024 threads (256 units of 4096
+// candidates run in one wave) or eight of 256 (1024 units of 1024 candidates do)
+template <int kSelThreads>
+__global__ void __launch_bounds__(kSelThreads, 2048 / kSelThreads)
 select_kernel(ModelView mv, BatchView bv, const float *scores, int *kept_idx, int *out_len, int smem_keys, int *status) {
+    constexpr int kSelWarps = kSelThreads / 32;
     extern __shared__ uint32_t key_cache[];  // the first min(N, smem_keys) keys
     __shared__ int hist[256];
     __shared__ int warp_tot[2][kSelWarps];
@@ -121,13 +124,13 @@ select_kernel(ModelView mv, BatchView bv, const float *scores, int *kept_idx, in
         if (lane == 31) buf[warp] = incl;
         __syncthreads();
         if (warp == 0) {
-            int t = buf[lane];
+            int t = lane < kSelWarps ? buf[lane] : 0;
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
                 const int up = __shfl_up_sync(0xffffffffu, t, off);
                 if (lane >= off) t += up;
             }
-            buf[lane] = t;  // inclusive totals of the warps
+            if (lane < kSelWarps) buf[lane] = t;  // inclusive totals of the warps
         }
         __syncthreads();
         total = buf[kSelWarps - 1];
@@ -200,12 +203,16 @@ cudaError_t launch_select(const Ctx &ctx, const float *scores, const BatchView &
     int smem_keys = max_n < 40960 ? max_n : 40960;  // up to 160 KiB of keys on chip; longer inputs re-read global
     if (smem_keys < 1) smem_keys = 1;
     const size_t smem = (size_t)smem_keys * sizeof(uint32_t);
-    cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
     dim3 grid(units, bv.batch);
     ctx.launches += 1;
-    return launch_chained(select_kernel, grid, dim3(kSelThreads), smem, stream, mv, bv, scores, (int *)kept_idx, out_len,
-                          smem_keys, ctx.d_status);
+    if (max_n <= 1024)
+        return launch_chained(select_kernel<kSelThreadsSmall>, grid, dim3(kSelThreadsSmall), smem, stream, mv, bv, scores,
+                              (int *)kept_idx, out_len, smem_keys, ctx.d_status);
+    cudaError_t e =
+        cudaFuncSetAttribute(select_kernel<kSelThreadsWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    return launch_chained(select_kernel<kSelThreadsWide>, grid, dim3(kSelThreadsWide), smem, stream, mv, bv, scores,
+                          (int *)kept_idx, out_len, smem_keys, ctx.d_status);
 }
 
 }  // namespace finch

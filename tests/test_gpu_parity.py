@@ -59,6 +59,10 @@ SHAPES = [
     # partial row blocks, partial key tiles on both sides of the cache/chunk seam
     ("bf16", 8, 2, 128, [(130, 9999, 300, 333)]),
     ("bf16", 4, 2, 64, [(64, 9999, 1, 129), (257, 9999, 257, 255), (40, 9999, 90, 70)]),
+    # single requests whose query rows fill three and two 128-row tiles per KV head (three heads x 100 rows: the
+    # tiles do not divide the four softmax groups; two heads x 100 rows: two groups per tile)
+    ("bf16", 6, 2, 64, [(100, 9999, 290, 260)]),
+    ("bf16", 4, 2, 128, [(100, 9999, 390, 270)]),
 ]
 
 
