@@ -88,6 +88,11 @@ __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
     return r;
 }
+__device__ __forceinline__ float4 lds128(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
 __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     uint64_t r;
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
@@ -178,7 +183,7 @@ __device__ __forceinline__ void lse_accumulate(uint32_t taddr, int valid, float 
 // Masked variant: lim2 holds, per pair of rows, how many candidates each row attends to; this thread's key has
 // candidate index j and counts for a row only if j is below that row's number.
 template <bool MASK>
-__device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[32], int nv, float scale2, const float4 *sm4, float &c0,
+__device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[32], int nv, float scale2, uint32_t sm4, float &c0,
                                              float &c1, const int2 *lim2, int j) {
     float v[32];
 #pragma unroll
@@ -191,7 +196,7 @@ __device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[32], int nv, fl
     uint64_t acc = pack2(c0, c1);
 #pragma unroll
     for (int e = 0; e < 32; e += 2) {
-        const float4 s4 = sm4[e / 2];  // two prompt rows: (-ref_a, -ref_b, w_a, w_b)
+        const float4 s4 = lds128(sm4 + (e / 2) * 16);  // two prompt rows: (-ref_a, -ref_b, w_a, w_b)
         float x0, x1;
         unpack2(fma2(pack2(v[e], v[e + 1]), s2, pack2(s4.x, s4.y)), x0, x1);
         if (MASK) {
@@ -207,7 +212,7 @@ __device__ __forceinline__ void colsum_chunk(const uint32_t (&r)[32], int nv, fl
 template <bool MASK>
 __device__ __forceinline__ void colsum_accumulate(uint32_t taddr, int v0, int v1, float scale2, const float2 *sm,
                                                   float &c0, float &c1, const int *lim, int j) {
-    const float4 *sm4 = (const float4 *)sm;
+    const uint32_t sm4 = smem_u32(sm);  // shared-window address: the loads below are ld.shared, not generic
     // chunks 0 and 1 cover the tile's first 64-row half (always present), chunks 2 and 3 the second half
     const int last = v1 > 0 ? 4 : 2;
 #pragma unroll 1
@@ -216,7 +221,7 @@ __device__ __forceinline__ void colsum_accumulate(uint32_t taddr, int v0, int v1
         __syncwarp();
         tmem_ld_x32_issue(taddr + cc * 32, r);
         tmem_ld_x32_wait(r);
-        colsum_chunk<MASK>(r, (cc < 2 ? v0 : v1) - (cc & 1) * 32, scale2, sm4 + cc * 16, c0, c1,
+        colsum_chunk<MASK>(r, (cc < 2 ? v0 : v1) - (cc & 1) * 32, scale2, sm4 + cc * 256, c0, c1,
                            (const int2 *)lim + cc * 16, j);
     }
 }

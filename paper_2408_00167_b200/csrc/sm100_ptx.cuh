@@ -34,17 +34,38 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait: polls (try_wait suspends the thread in hardware for a short while by itself) and gives up after
-// roughly a second, or as soon as another thread of the CTA has given up; it then raises *abort_flag and returns
-// false, and callers leave their loops for the common epilogue.  No software sleep on the fast path: a sleeping
-// waiter wakes too late for handshakes that complete in well under a microsecond.
-constexpr uint32_t kSpinLimit = 1u << 24;
+// The same test with a time limit for the hardware suspension: the thread sleeps inside the instruction until the
+// phase completes or about `ns` nanoseconds have passed, instead of coming back at once to poll again.
+__device__ __forceinline__ bool mbar_try_wait_for(uint64_t *bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  One plain test first (most barriers are complete when their waiter arrives); then tests that
+// suspend the thread in hardware, so that a waiting warp issues next to nothing -- a warp that polls in a tight
+// loop takes issue slots and shared-memory pipe cycles from the warps that compute on the same scheduler.  Gives
+// up after roughly a second of SM clocks, or soon after another thread of the CTA has given up; it then raises
+// *abort_flag and returns false, and callers leave their loops for the common epilogue.
+#ifndef FINCH_SUSPEND_NS
+#define FINCH_SUSPEND_NS 2000
+#endif
+constexpr uint32_t kSuspendNs = FINCH_SUSPEND_NS;
+constexpr long long kWaitClocks = 1ll << 31;
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 1023u) == 1023u) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait_for(bar, parity, kSuspendNs)) return true;
+        if ((it & 255u) == 0) {
             if (*abort_flag) return false;
-            if (it > (1u << 16)) __nanosleep(64);
+            if (clock64() - t0 > kWaitClocks) break;
         }
     }
     *abort_flag = 1;
