@@ -33,6 +33,11 @@ using namespace tc;
 // barriers, then the row statistics: 4 groups x 2 buffers x `tiles` query tiles
 constexpr int fused_aux_bytes(int tiles) { return 1024 + kGroups * 2 * tiles * kRows * 8; }
 constexpr int kSoftmaxWarps = kGroups * 4;
+// Waiters with time to spare poll rarely (their tests share the SM's memory-instruction queue with the softmax
+// warps' special-function instructions): the producer is a ring ahead of the MMAs, the helpers a window ahead of
+// anyone who needs what they publish.
+constexpr uint32_t kProducerSleepNs = 500;
+constexpr uint32_t kHelperSleepNs = 1000;
 constexpr int kHelpers = 64;  // two helper warps: the exchange of row statistics and the sum over the groups
 constexpr int kFusedThreads = kTcThreads + kHelpers;
 constexpr int kMaxSegs = 8;  // ranges that may overlap one unit (bounds the partial-statistics array)
@@ -86,7 +91,7 @@ __device__ __forceinline__ bool count_wait(int *counter, int target, volatile in
             return true;
         }
         if (*abort_flag) return false;
-        __nanosleep(64);
+        __nanosleep(kHelperSleepNs);
     }
     *abort_flag = 1;
     return false;
@@ -242,7 +247,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                         pst = 0;
                         pph ^= 1;
                     }
-                    if (!mbar_wait(&empty[stage], sph ^ 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait_relaxed(&empty[stage], sph ^ 1, abort_flag, kProducerSleepNs)) { ok = false; break; }
                     mbar_expect_tx(&full[stage], kTileBytes);
                     const KeyTile kt = key_tile(u, t);
                     const CUtensorMap *m = kt.is_chunk ? &chunk_map : &cache_map;

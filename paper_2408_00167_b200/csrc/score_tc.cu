@@ -231,7 +231,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                             pst = 0;
                             pph ^= 1;
                         }
-                        if (!mbar_wait(&empty[stage], ph ^ 1, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait_relaxed(&empty[stage], ph ^ 1, abort_flag, 500)) { ok = false; break; }
                         mbar_expect_tx(&full[stage], kTileBytes);
                         const KeyTile kt = key_tile(u, t);
                         const CUtensorMap *m = kt.is_chunk ? &chunk_map : &cache_map;

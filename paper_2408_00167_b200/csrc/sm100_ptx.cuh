@@ -72,6 +72,24 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     return false;
 }
 
+// The same for a waiter with time to spare (a producer far ahead of its consumers): it sleeps `ns` nanoseconds between
+// tests, so that its polling stays out of the way -- the tests, like the special-function instructions of the warps
+// that compute, go through the SM's memory-instruction queue.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint32_t ns) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        __nanosleep(ns);
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitClocks) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+
 // ---------------------------------------------------------------- TMA (tiled, 4-D, one destination CTA)
 __device__ __forceinline__ void tma_load_4d(void *smem_dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2,
                                             int c3) {
