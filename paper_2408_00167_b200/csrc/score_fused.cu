@@ -30,8 +30,8 @@ namespace {
 using namespace ptx;
 using namespace tc;
 
-// barriers, then the row statistics: 4 groups x 2 buffers x `tiles` query tiles
-constexpr int fused_aux_bytes(int tiles) { return 1024 + kGroups * 2 * tiles * kRows * 8; }
+// barriers, then the row statistics: 2 buffers x `tiles` query tiles
+constexpr int fused_aux_bytes(int tiles) { return 1024 + 2 * tiles * kRows * 8; }
 constexpr int kSoftmaxWarps = kGroups * 4;
 // Waiters with time to spare poll rarely (their tests share the SM's memory-instruction queue with the softmax
 // warps' special-function instructions): the producer is a ring ahead of the MMAs, the helpers a window ahead of
@@ -57,7 +57,6 @@ struct FusedParams {
     int stages;   // key-tile ring depth
     int q_tiles;  // resident query tiles (= query tiles of a unit, at most kQTiles)
     int delay;    // 0: phase B of a window right after its phase A; 1: one window later
-    int stats_tiles;  // room, in query tiles, of a softmax group's statistics buffer (3 when a unit can have 3 tiles)
 };
 
 __device__ __forceinline__ int ld_acquire_gpu(const int *p) {
@@ -142,14 +141,14 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     uint64_t *empty = full + kMaxStages;
     uint64_t *acc_full = empty + kMaxStages;
     uint64_t *acc_empty = acc_full + kAccBufs;
-    uint64_t *grp_ready = acc_empty + kAccBufs;  // [kGroups] the group's warps have staged their row statistics
-    uint32_t *tmem_slot = (uint32_t *)(grp_ready + kGroups);
+    uint64_t *stats_ready = acc_empty + kAccBufs;  // [2] the helper warps have staged a segment's row statistics
+    uint32_t *tmem_slot = (uint32_t *)(stats_ready + 2);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
     // Softmax warps -> helpers: plain counters (one count per warp and segment), not barrier phases, so that a helper
     // that falls behind by more than one segment still reads the right answer.
     int *a_count = (int *)(tmem_slot + 2);  // softmax warps that have written a phase-A segment's statistics
     int *b_count = a_count + 1;             // softmax warps that are through a phase-B segment
-    float2 *stats_sm = (float2 *)(aux + 1024);  // [kGroups][2][stats_tiles * 128] row statistics of phase B
+    float2 *stats_sm = (float2 *)(aux + 1024);  // [2][q_tiles * 128] row statistics of phase B, two segments in turn
 
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
@@ -164,7 +163,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             mbar_init(&acc_full[b], 1);
             mbar_init(&acc_empty[b], 4);  // one arrival per softmax warp of the owning group
         }
-        for (int b = 0; b < kGroups; ++b) mbar_init(&grp_ready[b], 4);
+        for (int b = 0; b < 2; ++b) mbar_init(&stats_ready[b], kHelpers / 32);  // one arrival per helper warp
         *a_count = 0;
         *b_count = 0;
         *abort_flag = 0;
@@ -319,10 +318,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const float scale2 = mv.scale * kLog2e;
         const int64_t cand = (int64_t)bv.total_cache + bv.total_chunk;
         const int64_t units = (int64_t)mv.L * mv.G;
-        const int gcd4 = (g.n_qt & 3) == 0 ? 4 : ((g.n_qt & 1) == 0 ? 2 : 1);  // gcd(query tiles, softmax groups)
-        // query tiles whose statistics this group stages: its own one when the tiles divide the groups, else all
-        const int st_tiles = g.n_qt > 0 && 4 % g.n_qt == 0 ? 1 : g.n_qt;
-        int A = 0, mine = 0, segs_b = 0, epoch = 0;
+        int A = 0, mine = 0, segs_b = 0;
         bool ok = true;
         FINCH_FOR_EACH_SEGMENT({
             if (ph == 0) {
@@ -379,60 +375,11 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 if (lane == 0) count_arrive(a_count);
             } else {
                 // ---------------------------------------------------------------- phase B: column sums
-                // all ranges of the unit have published their statistics once the ticket says so (with delay = 1
-                // that was a window ago)
-                int published = 1;
-                if (lane == 0) published = ticket_wait(&p.tickets[sg.unit], sg.n_seg, abort_flag);
-                if (!__shfl_sync(0xffffffffu, published, 0)) {
-                    ok = false;
-                    break;
-                }
-                // Each group merges and stages what its own accumulators will need -- one query tile when the tiles
-                // of a unit divide the four groups (its number is then fixed: accumulator A goes to group A % 4),
-                // all of them otherwise -- one row per thread, parts in a fixed order (ranges, then groups).  Only the
-                // group's four warps meet at the barrier, and they move in step anyway.  Two buffers: a warp past the
-                // barrier of epoch e has seen its group finish epoch e - 1, so the buffer of e + 1 is free.
-                float2 *sm_grp = stats_sm + ((grp * 2 + (epoch & 1)) * p.stats_tiles) * kRows;
-                {
-                    const float2 *part_stats = p.partial + ((int64_t)sg.unit * p.seg_max) * kGroups * p.rows_u;
-                    const int r = (sw & 3) * 32 + lane;  // this thread's row of the tile
-                    for (int qs = 0; qs < st_tiles; ++qs) {
-                        const int qb = st_tiles == 1 ? grp % g.n_qt : qs;
-                        const SubBlock sb = sub_block(2 * qb + r / kSub, g.sbq, g.n_sb, u.n_q);
-                        float2 out = make_float2(0.f, 0.f);
-                        if (qb < g.n_qt && r % kSub < sb.valid) {
-                            const int pr = sb.p0 + r % kSub;
-                            const float2 *src = part_stats + sb.hh * bv.max_q + pr;
-                            float M = -INFINITY, Z = 0.f;
-                            // group g' has met tile qb only if g' - qb is a multiple of gcd(tiles, groups)
-#pragma unroll 2
-                            for (int sgi = 0; sgi < sg.n_seg; ++sgi) {
-                                float2 part[kGroups];
-#pragma unroll
-                                for (int k = 0; k < kGroups; ++k)
-                                    part[k] = ((k - qb) & (gcd4 - 1)) == 0
-                                                  ? __ldcg(src + ((int64_t)sgi * kGroups + k) * p.rows_u)
-                                                  : make_float2(0.f, 0.f);
-#pragma unroll
-                                for (int k = 0; k < kGroups; ++k) merge_part(part[k], M, Z);
-                            }
-                            const int64_t row = ((int64_t)u.l * mv.Hq + u.G * mv.hpg + sb.hh) * bv.total_q + u.q0 + pr;
-                            if (bv.self_lse) merge_self_term(bv.self_lse[row], M, Z);
-                            float lse_nat;
-                            out = merged_pair(M, Z, lse_nat);
-                            // once per unit: its first range, and the one group whose number is the tile's
-                            if (p.row_lse && sg.slot == 0 && (st_tiles == 1 ? grp == qb : grp == 0)) p.row_lse[row] = lse_nat;
-                        }
-                        // rows 2k and 2k+1 share one float4: (-ref_2k, -ref_2k+1, w_2k, w_2k+1)
-                        float *smf = (float *)(sm_grp + qs * kRows) + (r >> 1) * 4 + (r & 1);
-                        smf[0] = out.x;
-                        smf[2] = out.y;
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&grp_ready[grp]);
-                    if (!__all_sync(0xffffffffu, mbar_wait(&grp_ready[grp], epoch & 1, abort_flag))) { ok = false; break; }
-                    ++epoch;
-                }
+                // The rows' merged statistics (-R, w) of this unit were staged by the helper warps while these warps ran
+                // the phase A that came in between; the barrier is normally complete.  Two buffers and two barriers
+                // in turn: the helpers cannot be two segments ahead, they wait for these warps' phase A in between.
+                if (!__all_sync(0xffffffffu, mbar_wait(&stats_ready[segs_b & 1], (segs_b >> 1) & 1, abort_flag))) { ok = false; break; }
+                const float2 *sm_seg = stats_sm + (segs_b & 1) * p.q_tiles * kRows;
                 float *part = p.score_parts + ((int64_t)grp * units + sg.unit) * cand + u.cache0 + u.chunk0;
                 for (int t = sg.t0; t < sg.t1 && ok; ++t) {
                     const KeyTile kt = key_tile(u, t);
@@ -445,7 +392,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                         tc_fence_after();
                         const int v0 = sub_block(2 * qb, g.sbq, g.n_sb, u.n_q).valid;
                         const int v1 = sub_block(2 * qb + 1, g.sbq, g.n_sb, u.n_q).valid;
-                        colsum_accumulate<false>(t_acc, v0, v1, scale2, sm_grp + (st_tiles == 1 ? 0 : qb) * kRows, c0, c1, nullptr, 0);
+                        colsum_accumulate<false>(t_acc, v0, v1, scale2, sm_seg + qb * kRows, c0, c1, nullptr, 0);
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&acc_empty[grp]);
@@ -468,18 +415,65 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const int tid = threadIdx.x - (2 + kSoftmaxWarps) * 32;
         const int64_t cand = (int64_t)bv.total_cache + bv.total_chunk;
         const int64_t units = (int64_t)mv.L * mv.G;
+        const int gcd4 = (g.n_qt & 3) == 0 ? 4 : ((g.n_qt & 1) == 0 ? 2 : 1);  // gcd(query tiles, softmax groups)
         int segs_a = 0, segs_b = 0;
         bool ok = true;
         auto warp_agree = [&](bool good) -> bool { return __all_sync(0xffffffffu, good); };
         FINCH_FOR_EACH_SEGMENT({
             if (ph == 0) {
                 ++segs_a;
-                if (tid >= 32) continue;  // the first helper warp's business
+                // every softmax warp has written the segment's statistics (and is through the phase B of two
+                // segments ago, whose buffer is reused below)
                 if (!warp_agree(lane != 0 || count_wait(a_count, kSoftmaxWarps * segs_a, abort_flag))) { ok = false; break; }
-                if (lane == 0) {
+                if (tid == 0) {
                     __threadfence();  // cumulative: covers the softmax warps' stores this thread has synchronised with
                     atomicAdd(&p.tickets[sg.unit], 1);
                 }
+                // Stage the unit's statistics for the segment's phase B, which the softmax warps reach one phase A
+                // later: wait (bounded) until every range of the unit has published -- the other ranges belong to
+                // neighbouring CTAs that run the same window at the same time -- then merge the parts of each prompt
+                // row in a fixed order (ranges, then groups) into (-R, w).
+                int published = 1;
+                if (lane == 0) published = ticket_wait(&p.tickets[sg.unit], sg.n_seg, abort_flag);
+                if (!__shfl_sync(0xffffffffu, published, 0)) {
+                    ok = false;
+                    break;
+                }
+                float2 *sm_seg = stats_sm + ((segs_a - 1) & 1) * p.q_tiles * kRows;
+                const float2 *part_stats = p.partial + ((int64_t)sg.unit * p.seg_max) * kGroups * p.rows_u;
+                for (int i = tid; i < g.n_qt * kRows; i += kHelpers) {
+                    const int qb = i / kRows, r = i % kRows;  // query tile, row of the tile
+                    const SubBlock sb = sub_block(2 * qb + r / kSub, g.sbq, g.n_sb, u.n_q);
+                    float2 out = make_float2(0.f, 0.f);
+                    if (r % kSub < sb.valid) {
+                        const int pr = sb.p0 + r % kSub;
+                        const float2 *src = part_stats + sb.hh * bv.max_q + pr;
+                        float M = -INFINITY, Z = 0.f;
+                        // group g' has met tile qb only if g' - qb is a multiple of gcd(tiles, groups)
+#pragma unroll 2
+                        for (int sgi = 0; sgi < sg.n_seg; ++sgi) {
+                            float2 part[kGroups];
+#pragma unroll
+                            for (int k = 0; k < kGroups; ++k)
+                                part[k] = ((k - qb) & (gcd4 - 1)) == 0
+                                              ? __ldcg(src + ((int64_t)sgi * kGroups + k) * p.rows_u)
+                                              : make_float2(0.f, 0.f);
+#pragma unroll
+                            for (int k = 0; k < kGroups; ++k) merge_part(part[k], M, Z);
+                        }
+                        const int64_t row = ((int64_t)u.l * mv.Hq + u.G * mv.hpg + sb.hh) * bv.total_q + u.q0 + pr;
+                        if (bv.self_lse) merge_self_term(bv.self_lse[row], M, Z);
+                        float lse_nat;
+                        out = merged_pair(M, Z, lse_nat);
+                        if (p.row_lse && sg.slot == 0) p.row_lse[row] = lse_nat;  // once per unit: by its first range
+                    }
+                    // rows 2k and 2k+1 share one float4: (-ref_2k, -ref_2k+1, w_2k, w_2k+1)
+                    float *smf = (float *)(sm_seg + qb * kRows) + (r >> 1) * 4 + (r & 1);
+                    smf[0] = out.x;
+                    smf[2] = out.y;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&stats_ready[(segs_a - 1) & 1]);
             } else {
                 ++segs_b;
                 if (!warp_agree(lane != 0 || count_wait(b_count, kSoftmaxWarps * segs_b, abort_flag))) { ok = false; break; }
@@ -576,7 +570,7 @@ cudaError_t launch_fused_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensor
     constexpr int kTileBytes = (D / 64) * kSlabBytes;
     const ModelView &mv = p.mv;
     const BatchView &bv = p.bv;
-    const int aux = fused_aux_bytes(p.stats_tiles);
+    const int aux = fused_aux_bytes(p.q_tiles);
     p.stages = min(kMaxStages, (kSmemLimit - 1024 - aux - p.q_tiles * kTileBytes) / kTileBytes);
     if (p.stages < 2) return cudaErrorNotSupported;
     const int smem = 1024 + (p.q_tiles + p.stages) * kTileBytes + aux;
@@ -650,7 +644,6 @@ cudaError_t launch_score_fused(const Ctx &ctx, const TensorView &q, const Tensor
     p.rows_u = mv.g * bv.max_q;
     p.q_tiles = (mv.g * ((bv.max_q + kSub - 1) / kSub) + 1) / 2;
     p.delay = 1;
-    p.stats_tiles = p.q_tiles >= 3 ? 3 : 1;  // a unit with three tiles (4 % 3 != 0) stages all of them per group
     if (p.W == 0) return cudaErrorNotSupported;
     const int n_ranges = (int)(((long long)units * tiles + p.W - 1) / p.W);
     return mv.d == 64 ? launch_fused_d<64>(ctx, qm, cm, hm, p, n_ranges, ctx.model.G, ctx.model.kvpg, scores, stream)
