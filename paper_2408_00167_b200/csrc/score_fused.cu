@@ -136,8 +136,9 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     uint8_t *q_res = smem;
     uint8_t *k_ring = smem + p.q_tiles * kTileBytes;
     uint8_t *aux = k_ring + p.stages * kTileBytes;
-    uint64_t *q_full = (uint64_t *)aux;
-    uint64_t *full = q_full + 1;
+    uint64_t *q_full = (uint64_t *)aux;    // [kQTiles] a query tile of the segment's unit has landed
+    uint64_t *q_free = q_full + kQTiles;   // [kQTiles] the segment's MMAs are through with a query tile
+    uint64_t *full = q_free + kQTiles;
     uint64_t *empty = full + kMaxStages;
     uint64_t *acc_full = empty + kMaxStages;
     uint64_t *acc_empty = acc_full + kAccBufs;
@@ -154,7 +155,10 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const BatchView &bv = p.bv;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        mbar_init(q_full, 1);
+        for (int b = 0; b < kQTiles; ++b) {
+            mbar_init(&q_full[b], 1);
+            mbar_init(&q_free[b], 1);
+        }
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
@@ -220,47 +224,54 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             prefetch_tensormap(&q_map);
             prefetch_tensormap(&cache_map);
             prefetch_tensormap(&chunk_map);
-            int kcnt = 0, qcnt = 0, pst = 0, pph = 0, last_stage = 0, last_ph = 0, prev_stage = 0, prev_ph = 0, q_unit = -1;
+            int kcnt = 0, qcnt = 0, nseg = 0, pst = 0, pph = 0, q_unit = -1;
             bool ok = true;
+            auto load_key_tile = [&](const UnitInfo &u, int t) {
+                const int stage = pst, sph = pph;
+                if (++pst == p.stages) {
+                    pst = 0;
+                    pph ^= 1;
+                }
+                if (!mbar_wait_relaxed(&empty[stage], sph ^ 1, abort_flag, kProducerSleepNs)) {
+                    ok = false;
+                    return;
+                }
+                mbar_expect_tx(&full[stage], kTileBytes);
+                const KeyTile kt = key_tile(u, t);
+                const CUtensorMap *m = kt.is_chunk ? &chunk_map : &cache_map;
+                for (int s = 0; s < kSlabs; ++s)
+                    tma_load_4d(k_ring + stage * kTileBytes + s * kSlabBytes, m, &full[stage], s * 64, kt.row0, u.G, u.l);
+                ++kcnt;
+            };
             FINCH_FOR_EACH_SEGMENT({
+                // the segment's first key tile goes first: its ring stage is free before the query tiles are
+                load_key_tile(u, sg.t0);
+                if (!ok) break;
                 if (q_unit != sg.unit) {
-                    // every MMA issued so far must have read the resident query tiles: wait for the release of the
-                    // last two key tiles loaded
-                    if (kcnt > 1 && !mbar_wait(&empty[prev_stage], prev_ph, abort_flag)) { ok = false; break; }
-                    if (kcnt > 0 && !mbar_wait(&empty[last_stage], last_ph, abort_flag)) { ok = false; break; }
-                    const int nload = min(2 * g.n_qt, g.n_sb);
-                    mbar_expect_tx(q_full, nload * kSlabs * kSubBytes);
-                    for (int sl = 0; sl < nload; ++sl) {
-                        const SubBlock sb = sub_block(sl, g.sbq, g.n_sb, u.n_q);
-                        uint8_t *dst = q_res + (sl / 2) * kTileBytes + (sl % 2) * kSubBytes;
-                        for (int s = 0; s < kSlabs; ++s)
-                            tma_load_4d(dst + s * kSlabBytes, &q_map, q_full, s * 64, u.q0 + sb.p0, u.G * mv.hpg + sb.hh,
-                                        u.l);
+                    // Another unit's query tiles, one tile at a time: tile qb may be overwritten once the previous
+                    // segment's last MMAs on it are complete (its q_free phase), while the MMAs on the tiles behind it
+                    // still run -- the reload hides behind the tail of the old segment instead of following it.
+                    for (int qb = 0; qb < g.n_qt; ++qb) {
+                        if (nseg > 0 && !mbar_wait(&q_free[qb], (nseg - 1) & 1, abort_flag)) { ok = false; break; }
+                        const int nsb = min(2, g.n_sb - 2 * qb);
+                        mbar_expect_tx(&q_full[qb], nsb * kSlabs * kSubBytes);
+                        for (int sl = 2 * qb; sl < 2 * qb + nsb; ++sl) {
+                            const SubBlock sb = sub_block(sl, g.sbq, g.n_sb, u.n_q);
+                            uint8_t *dst = q_res + (sl / 2) * kTileBytes + (sl % 2) * kSubBytes;
+                            for (int s = 0; s < kSlabs; ++s)
+                                tma_load_4d(dst + s * kSlabBytes, &q_map, &q_full[qb], s * 64, u.q0 + sb.p0,
+                                            u.G * mv.hpg + sb.hh, u.l);
+                        }
                     }
+                    if (!ok) break;
                     ++qcnt;
                     q_unit = sg.unit;
                 }
-                for (int t = sg.t0; t < sg.t1; ++t, ++kcnt) {
-                    const int stage = pst, sph = pph;
-                    if (++pst == p.stages) {
-                        pst = 0;
-                        pph ^= 1;
-                    }
-                    if (!mbar_wait_relaxed(&empty[stage], sph ^ 1, abort_flag, kProducerSleepNs)) { ok = false; break; }
-                    mbar_expect_tx(&full[stage], kTileBytes);
-                    const KeyTile kt = key_tile(u, t);
-                    const CUtensorMap *m = kt.is_chunk ? &chunk_map : &cache_map;
-                    for (int s = 0; s < kSlabs; ++s)
-                        tma_load_4d(k_ring + stage * kTileBytes + s * kSlabBytes, m, &full[stage], s * 64, kt.row0, u.G,
-                                    u.l);
-                    prev_stage = last_stage;
-                    prev_ph = last_ph;
-                    last_stage = stage;
-                    last_ph = sph;
-                }
+                ++nseg;
+                for (int t = sg.t0 + 1; t < sg.t1 && ok; ++t) load_key_tile(u, t);
             })
             // no copy may still be in flight when the CTA retires: wait (bounded) for the last loads issued
-            if (qcnt) mbar_wait(q_full, (qcnt - 1) & 1, abort_flag);
+            for (int qb = 0; qcnt && qb < g.n_qt; ++qb) mbar_wait(&q_full[qb], (qcnt - 1) & 1, abort_flag);
             for (int i = max(0, kcnt - p.stages); i < kcnt; ++i)
                 mbar_wait(&full[i % p.stages], (i / p.stages) & 1, abort_flag);
         }
@@ -272,17 +283,15 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             bool ok = true;
             int A = 0, qcnt = 0, q_unit = -1, st = 0, sph = 0;
             FINCH_FOR_EACH_SEGMENT({
-                if (q_unit != sg.unit) {
-                    if (!mbar_wait(q_full, qcnt & 1, abort_flag)) { ok = false; break; }
-                    ++qcnt;
-                    q_unit = sg.unit;
-                }
+                const bool reloaded = q_unit != sg.unit;  // the producer has brought this unit's query tiles
+                q_unit = sg.unit;
                 for (int t = sg.t0; t < sg.t1 && ok; ++t) {
                     if (!mbar_wait(&full[st], sph, abort_flag)) { ok = false; break; }
                     const uint64_t kd = ring_desc + (uint64_t)((st * kTileBytes) >> 4);
                     for (int qb = 0; qb < g.n_qt; ++qb, ++A) {
                         const int buf = A & 3;
                         if (!mbar_wait(&acc_empty[buf], ((A >> 2) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                        if (reloaded && t == sg.t0 && !mbar_wait(&q_full[qb], qcnt & 1, abort_flag)) { ok = false; break; }
                         tc_fence_after();
                         // phase A: prompt rows on the lanes (A = query tile); phase B: keys on the lanes (A = key tile)
                         const uint64_t qd = q_desc + (uint64_t)((qb * kTileBytes) >> 4);
@@ -297,6 +306,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                                 umma_bf16_acc(d_addr, a_desc + off, b_desc + off, idesc);
                         }
                         umma_commit(&acc_full[buf]);
+                        if (t == sg.t1 - 1) umma_commit(&q_free[qb]);  // the segment is through with this query tile
                     }
                     if (ok) umma_commit(&empty[st]);  // the stage may be refilled once these MMAs have read it
                     if (++st == p.stages) {
@@ -304,6 +314,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                         sph ^= 1;
                     }
                 }
+                if (reloaded) ++qcnt;
             })
         }
     } else if (warp < 2 + kSoftmaxWarps) {
