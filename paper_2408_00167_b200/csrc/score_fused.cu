@@ -461,7 +461,7 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                         const float2 *src = part_stats + sb.hh * bv.max_q + pr;
                         float M = -INFINITY, Z = 0.f;
                         // group g' has met tile qb only if g' - qb is a multiple of gcd(tiles, groups)
-#pragma unroll 2
+#pragma unroll 4
                         for (int sgi = 0; sgi < sg.n_seg; ++sgi) {
                             float2 part[kGroups];
 #pragma unroll
