@@ -331,23 +331,34 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const int64_t units = (int64_t)mv.L * mv.G;
         int A = 0, mine = 0, segs_b = 0;
         bool ok = true;
+        // What depends on the geometry only (the same for every unit of a single-request batch) is worked out once:
+        // between two accumulators a softmax warp shares its scheduler's issue slots with three warps that compute,
+        // so every instruction of bookkeeping there costs about four cycles.
+        uint32_t live_mask = 0;   // bit qb: this thread's row of query tile qb holds a prompt row
+        uint64_t valid_pack = 0;  // byte 2 qb / 2 qb + 1: prompt rows in the first / second 64-row half of tile qb
+#pragma unroll
+        for (int k = 0; k < kQTiles; ++k) {
+            const SubBlock sb = sub_block(2 * k + my_row / kSub, g.sbq, g.n_sb, g.u.n_q);
+            if (k < g.n_qt && my_row % kSub < sb.valid) live_mask |= 1u << k;
+            valid_pack |= (uint64_t)sub_block(2 * k, g.sbq, g.n_sb, g.u.n_q).valid << (16 * k);
+            valid_pack |= (uint64_t)sub_block(2 * k + 1, g.sbq, g.n_sb, g.u.n_q).valid << (16 * k + 8);
+        }
         FINCH_FOR_EACH_SEGMENT({
             if (ph == 0) {
                 // ---------------------------------------------------------------- phase A: row statistics
                 float m_raw[kQTiles], z[kQTiles];
-                uint32_t live_mask = 0;  // bit qb: this thread's row of query tile qb holds a prompt row
 #pragma unroll
                 for (int k = 0; k < kQTiles; ++k) {
                     m_raw[k] = -INFINITY;
                     z[k] = 0.f;
-                    const SubBlock sb = sub_block(2 * k + my_row / kSub, g.sbq, g.n_sb, u.n_q);
-                    if (k < g.n_qt && my_row % kSub < sb.valid) live_mask |= 1u << k;
                 }
                 for (int t = sg.t0; t < sg.t1 && ok; ++t) {
                     const KeyTile kt = key_tile(u, t);
-#pragma unroll 1
-                    for (int qb = 0; qb < g.n_qt && ok; ++qb, ++A) {
-                        if ((A & 3) != grp) continue;  // another group's accumulator
+                    // the one accumulator of this key tile that belongs to the group, if any (accumulator A goes to
+                    // group A % 4, a key tile has at most four)
+                    const int qb = (grp - A) & 3;
+                    A += g.n_qt;
+                    if (qb < g.n_qt) {
                         // a wait's verdict is made warp-uniform so that a timeout takes the whole warp out
                         if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[grp], mine & 1, abort_flag))) { ok = false; break; }
                         ++mine;
@@ -395,14 +406,13 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 for (int t = sg.t0; t < sg.t1 && ok; ++t) {
                     const KeyTile kt = key_tile(u, t);
                     float c0 = 0.f, c1 = 0.f;
-#pragma unroll 1
-                    for (int qb = 0; qb < g.n_qt && ok; ++qb, ++A) {
-                        if ((A & 3) != grp) continue;
+                    const int qb = (grp - A) & 3;
+                    A += g.n_qt;
+                    if (qb < g.n_qt) {
                         if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[grp], mine & 1, abort_flag))) { ok = false; break; }
                         ++mine;
                         tc_fence_after();
-                        const int v0 = sub_block(2 * qb, g.sbq, g.n_sb, u.n_q).valid;
-                        const int v1 = sub_block(2 * qb + 1, g.sbq, g.n_sb, u.n_q).valid;
+                        const int v0 = (int)(valid_pack >> (16 * qb)) & 0xff, v1 = (int)(valid_pack >> (16 * qb + 8)) & 0xff;
                         colsum_accumulate<false>(t_acc, v0, v1, scale2, sm_seg + qb * kRows, c0, c1, nullptr, 0);
                         tc_fence_before();
                         __syncwarp();
