@@ -559,9 +559,10 @@ sum_heads_kernel(ModelView mv, BatchView bv, const float *unit_scores, float *sc
 // Key tiles per range, or 0 when the one-kernel path should leave the batch to the two-launch kernels.  A range
 // divides the unit's tiles (otherwise ranges straddle units: the query tiles change inside a range and a unit's tiles
 // are dealt unevenly), is long enough to amortise a window's fixed costs (query loads, the exchange of the row
-// statistics: at least four tiles, or the whole unit), short enough that the keys in flight between a window's sweeps stay in L2, and fills the last window
-// of the persistent grid to at least 90 %.  Where no such length exists the two-launch kernels, whose key splits are
-// chosen per launch, were the faster ones (27 tiles per unit, 256 units: 0.270 against 0.282 - 0.291 ms per step).
+// statistics: at least four tiles, or the whole unit), short enough that the keys in flight between a window's sweeps
+// stay in L2, and fills the CTA x window slots of the persistent grid to at least 85 % (27 tiles per unit, 256 units:
+// windows of 9 fill 86 % and the step takes 0.258 ms against 0.261 on the two-launch kernels, with K read once).
+// Where no such length exists the batch goes to the two-launch kernels, whose key splits are chosen per launch.
 int choose_window(long long units, int tiles_per_unit, int ctas, int tile_bytes) {
     const long long total = units * tiles_per_unit;
     const long long l2_budget = 40ll << 20;
@@ -574,7 +575,7 @@ int choose_window(long long units, int tiles_per_unit, int ctas, int tile_bytes)
         if (W > 1 && (long long)W * ctas * tile_bytes > l2_budget && best) break;
         const long long ranges = total / W, windows = (ranges + ctas - 1) / ctas;
         const double fill = (double)total / (double)(windows * W * (ranges < ctas ? ranges : ctas));
-        if (fill < 0.9) continue;
+        if (fill < 0.85) continue;
         const double score = fill - 0.04 / W;
         if (score > best_score) {
             best_score = score;
