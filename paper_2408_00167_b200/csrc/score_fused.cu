@@ -280,33 +280,45 @@ score_fused_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_bf16_f32(kRows, kRows);
             const uint64_t q_desc = smem_desc_sw128(smem_u32(q_res)), ring_desc = smem_desc_sw128(smem_u32(k_ring));
+            const uint32_t desc_hi = (uint32_t)(q_desc >> 32), q_lo = (uint32_t)q_desc, ring_lo = (uint32_t)ring_desc;
             bool ok = true;
             int A = 0, qcnt = 0, q_unit = -1, st = 0, sph = 0;
             FINCH_FOR_EACH_SEGMENT({
                 const bool reloaded = q_unit != sg.unit;  // the producer has brought this unit's query tiles
                 q_unit = sg.unit;
+                // This thread is the kernel's pacemaker (it is held while its MMAs run and every barrier test costs
+                // it some 200 cycles), so its loop carries as little as possible: descriptor bases and strides are
+                // set per segment -- phase A: A operand = query tile qb, B = the key tile; phase B the other way
+                // round -- and the MMAs' operands differ in their low words only (the 14-bit address field cannot
+                // carry: shared memory ends below 2^18 bytes).
+                const uint32_t q_step = (uint32_t)(kTileBytes >> 4), k_step = (uint32_t)(kTileBytes >> 4);
+                const uint32_t a_q = ph == 0 ? q_step : 0u, a_k = ph == 0 ? 0u : k_step;  // strides of the A operand
+                const uint32_t b_q = ph == 0 ? 0u : q_step, b_k = ph == 0 ? k_step : 0u;  // and of the B operand
+                const uint32_t a_lo0 = ph == 0 ? q_lo : ring_lo, b_lo0 = ph == 0 ? ring_lo : q_lo;
+                const bool wait_q = reloaded;
                 for (int t = sg.t0; t < sg.t1 && ok; ++t) {
                     if (!mbar_wait(&full[st], sph, abort_flag)) { ok = false; break; }
-                    const uint64_t kd = ring_desc + (uint64_t)((st * kTileBytes) >> 4);
+                    const bool first = wait_q && t == sg.t0, last = t == sg.t1 - 1;
                     for (int qb = 0; qb < g.n_qt; ++qb, ++A) {
                         const int buf = A & 3;
                         if (!mbar_wait(&acc_empty[buf], ((A >> 2) & 1) ^ 1, abort_flag)) { ok = false; break; }
-                        if (reloaded && t == sg.t0 && !mbar_wait(&q_full[qb], qcnt & 1, abort_flag)) { ok = false; break; }
+                        if (first && !mbar_wait(&q_full[qb], qcnt & 1, abort_flag)) { ok = false; break; }
                         tc_fence_after();
-                        // phase A: prompt rows on the lanes (A = query tile); phase B: keys on the lanes (A = key tile)
-                        const uint64_t qd = q_desc + (uint64_t)((qb * kTileBytes) >> 4);
-                        const uint64_t a_desc = ph == 0 ? qd : kd, b_desc = ph == 0 ? kd : qd;
+                        const uint32_t a_lo = a_lo0 + (uint32_t)qb * a_q + (uint32_t)st * a_k;
+                        const uint32_t b_lo = b_lo0 + (uint32_t)qb * b_q + (uint32_t)st * b_k;
                         const uint32_t d_addr = tmem_base + buf * kRows;
 #pragma unroll
                         for (int k = 0; k < D / 16; ++k) {
-                            const uint64_t off = (uint64_t)(((k / 4) * kSlabBytes + (k % 4) * 32) >> 4);
+                            const uint32_t off = (uint32_t)(((k / 4) * kSlabBytes + (k % 4) * 32) >> 4);
+                            const uint64_t a_desc = ((uint64_t)desc_hi << 32) | (a_lo + off);
+                            const uint64_t b_desc = ((uint64_t)desc_hi << 32) | (b_lo + off);
                             if (k == 0)
-                                umma_bf16_first(d_addr, a_desc + off, b_desc + off, idesc);
+                                umma_bf16_first(d_addr, a_desc, b_desc, idesc);
                             else
-                                umma_bf16_acc(d_addr, a_desc + off, b_desc + off, idesc);
+                                umma_bf16_acc(d_addr, a_desc, b_desc, idesc);
                         }
                         umma_commit(&acc_full[buf]);
-                        if (t == sg.t1 - 1) umma_commit(&q_free[qb]);  // the segment is through with this query tile
+                        if (last) umma_commit(&q_free[qb]);  // the segment is through with this query tile
                     }
                     if (ok) umma_commit(&empty[st]);  // the stage may be refilled once these MMAs have read it
                     if (++st == p.stages) {
