@@ -168,6 +168,23 @@ finch_status finch_score(finch_ctx *ctx, const finch_tensor *prompt_q, const fin
                          const finch_tensor *chunk_k, const finch_batch *batch, float *scores, float *row_lse,
                          void *ws, size_t ws_bytes, void *cuda_stream);
 
+/* Which kernels finch_score and finch_step run for a batch (given a workspace of finch_workspace_bytes).  Host
+ * arithmetic, nothing is enqueued, works on a validation-only context.  (The paper prescribes no kernel; this is how
+ * its prompt x candidate block, Section "Method", is tiled here.)
+ *  - FINCH_SCORE_ONE_KERNEL: bf16, head_dim 64 or 128, a single request without row_limit, at most four 128-row
+ *    query tiles per KV head (queries per KV head x ceil(prompt rows / 64) <= 8), and a window length for its key
+ *    tiles exists: a divisor W of the tiles per (layer, KV head) unit with W >= 4 (or the whole unit),
+ *    tiles / W <= 8, W x SMs x tile bytes <= 40 MiB, and the persistent grid's CTA x window slots >= 85 % full.
+ *    *window receives W (key tiles of 128 candidates).  Both sweeps of the softmax run in one persistent kernel.
+ *  - FINCH_SCORE_TWO_LAUNCH: bf16, head_dim 64 or 128 otherwise (several requests, causal rows, longer prompts, no
+ *    usable window): row statistics and column sums in two tensor-core launches.  *window = 0.
+ *  - FINCH_SCORE_WARP_LEVEL: fp32 inputs or another head_dim.  *window = 0.
+ * A batch whose tensors the TMA unit cannot describe (an outer stride of 2^40 bytes or more) takes the warp-level
+ * kernels regardless; that depends on the tensors, not on the batch, and is not reported here.
+ * `window` may be NULL.  Errors: as finch_workspace_bytes. */
+enum { FINCH_SCORE_WARP_LEVEL = 0, FINCH_SCORE_TWO_LAUNCH = 1, FINCH_SCORE_ONE_KERNEL = 2 };
+finch_status finch_score_plan(const finch_ctx *ctx, const finch_batch *batch, int32_t *path, int32_t *window);
+
 /* The same scores and row_lse as finch_score, for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is an integration aid.)  Some hosts of this library may not call cudaMalloc at all -- a plugin
  * inside a serving process whose memory pool owns the whole device, or a step that must stay clear of the driver's

@@ -33,7 +33,7 @@ FINCH_DEV_BAD_BATCH, FINCH_DEV_TIMEOUT, FINCH_DEV_BAD_INDEX = 1, 2, 4
 
 EXPORTS = ("finch_ctx_create", "finch_ctx_destroy", "finch_workspace_bytes", "finch_score", "finch_select",
            "finch_compact", "finch_step", "finch_device_status", "finch_launch_count", "finch_status_string", "finch_score_static", "finch_score_static_max_rows", "finch_score_static_path",
-           "finch_step_host")
+           "finch_step_host", "finch_score_plan")
 
 
 class finch_config(C.Structure):
@@ -238,6 +238,17 @@ def finch_score_static(ctx, prompt_q, cache_k, chunk_k, batch: Batch, scores, ro
 
 def finch_score_static_max_rows() -> int:
     return int(load().finch_score_static_max_rows())
+
+
+FINCH_SCORE_WARP_LEVEL, FINCH_SCORE_TWO_LAUNCH, FINCH_SCORE_ONE_KERNEL = 0, 1, 2
+
+
+def finch_score_plan(ctx, batch: Batch):
+    """(path, window): which kernels finch_score / finch_step run for this batch and, on the one-kernel path, the
+    window length in key tiles."""
+    path, window = C.c_int32(), C.c_int32()
+    _check(load().finch_score_plan(ctx, C.byref(batch.c), C.byref(path), C.byref(window)), "finch_score_plan")
+    return path.value, window.value
 
 
 def finch_score_static_path(ctx, batch: Batch) -> bool:

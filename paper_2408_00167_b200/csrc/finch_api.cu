@@ -526,6 +526,18 @@ extern "C" size_t finch_score_static_max_rows(void) { return kStaticRows; }
 // Which kernels finch_score_static runs for a batch: the tensor-core kernels keep more than one entry per prompt row
 // in the scratch (statistics per key range and softmax group, partial column sums per candidate), so a batch can
 // fit the array's row limit and still be too large for them; it then takes the warp-level kernels.
+// Which kernels finch_score / finch_step run for a batch (workspace of finch_workspace_bytes): see the header.
+extern "C" finch_status finch_score_plan(const finch_ctx *ctx, const finch_batch *batch, int32_t *path, int32_t *window) {
+    if (!path) return FINCH_ERR_INVALID_ARG;
+    finch_status s = check_batch(ctx, batch);
+    if (s) return s;
+    const BatchView bv = view_of(batch);
+    const int w = score_fused_window(*ctx, bv);
+    *path = w > 0 ? FINCH_SCORE_ONE_KERNEL : (score_tc_supported(*ctx) ? FINCH_SCORE_TWO_LAUNCH : FINCH_SCORE_WARP_LEVEL);
+    if (window) *window = w;
+    return FINCH_OK;
+}
+
 extern "C" finch_status finch_score_static_path(const finch_ctx *ctx, const finch_batch *batch, int32_t *tensor_cores) {
     if (!tensor_cores) return FINCH_ERR_INVALID_ARG;
     finch_status s = check_batch(ctx, batch);

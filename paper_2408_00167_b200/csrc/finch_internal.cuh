@@ -141,6 +141,7 @@ cudaError_t launch_score_tc(const Ctx &ctx, const TensorView &q, const TensorVie
 // both sweeps in one persistent kernel (single-request batches without a row mask whose query tiles fit the shared
 // memory): score_fused_scratch gives the float2 entries of scratch it needs, 0 when it does not take the batch
 size_t score_fused_scratch(const Ctx &ctx, const BatchView &bv);
+int score_fused_window(const Ctx &ctx, const BatchView &bv);  // key tiles per window; 0: the batch goes elsewhere
 cudaError_t launch_score_fused(const Ctx &ctx, const TensorView &q, const TensorView &cache_k, const TensorView &chunk_k,
                                const BatchView &bv, float *scores, float2 *scratch, size_t scratch_capacity,
                                float *row_lse, cudaStream_t stream);

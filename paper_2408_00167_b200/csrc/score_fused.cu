@@ -626,13 +626,22 @@ cudaError_t launch_fused_d(const Ctx &ctx, const CUtensorMap &qm, const CUtensor
 
 }  // namespace
 
-// Float2 entries of scratch the fused kernel needs for this batch (0: the batch is not one it takes).
-size_t score_fused_scratch(const Ctx &ctx, const BatchView &bv) {
+// Key tiles per window the fused kernel would use for this batch; 0: the batch is not one it takes (several
+// requests, causal rows, more than four query tiles per KV head, no window length that fits: see choose_window).
+int score_fused_window(const Ctx &ctx, const BatchView &bv) {
     const ModelView &mv = ctx.model;
     if (!score_tc_supported(ctx) || bv.batch != 1 || bv.row_limit || bv.max_q == 0 || bv.max_cache + bv.max_chunk == 0)
         return 0;
     const int sub_blocks = mv.g * ((bv.max_q + kSub - 1) / kSub);
     if ((sub_blocks + 1) / 2 > kQTiles) return 0;
+    const int tiles = (bv.max_cache + kRows - 1) / kRows + (bv.max_chunk + kRows - 1) / kRows;
+    return choose_window((long long)mv.L * mv.Hkv, tiles, ctx.sm_count > 0 ? ctx.sm_count : 148, (mv.d / 64) * kSlabBytes);
+}
+
+// Float2 entries of scratch the fused kernel needs for this batch (0: the batch is not one it takes).
+size_t score_fused_scratch(const Ctx &ctx, const BatchView &bv) {
+    const ModelView &mv = ctx.model;
+    if (score_fused_window(ctx, bv) == 0) return 0;
     const size_t rows = (size_t)mv.L * mv.Hq * (size_t)bv.max_q;
     const size_t units = (size_t)mv.L * mv.Hkv, cand = (size_t)bv.total_cache + bv.total_chunk;
     size_t n = rows * kMaxSegs * kGroups;      // partial row statistics
@@ -673,7 +682,7 @@ cudaError_t launch_score_fused(const Ctx &ctx, const TensorView &q, const Tensor
     p.unit_scores = ctx.model.G == mv.Hkv ? scores : p.score_parts + (((size_t)kGroups * units * cand + 1) & ~(size_t)1);
     p.row_lse = row_lse;
     p.status = ctx.d_status;
-    p.W = choose_window(units, tiles, sms, (mv.d / 64) * kSlabBytes);
+    p.W = score_fused_window(ctx, bv);
     p.seg_max = kMaxSegs;
     p.rows_u = mv.g * bv.max_q;
     p.q_tiles = (mv.g * ((bv.max_q + kSub - 1) / kSub) + 1) / 2;

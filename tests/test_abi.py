@@ -202,3 +202,49 @@ def test_step_host_validation(lib):
         assert call(ws_bytes=1024) == fb.FINCH_ERR_WORKSPACE_TOO_SMALL
     finally:
         fb.finch_ctx_destroy(ctx)
+
+
+# ---------------------------------------------------------------------------------------------- the score plan
+
+def _plan(n_layers, n_q_heads, n_kv_heads, head_dim, n_q, cache, chunk, dtype=None, requests=1, row_limit=None):
+    dtype = fb.FINCH_BF16 if dtype is None else dtype
+    ctx = fb.finch_ctx_create(n_layers=n_layers, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, head_dim=head_dim,
+                              dtype=dtype, group_mode=fb.FINCH_GROUP_PER_KV_HEAD, scale=0.0, max_batch=requests,
+                              max_prompt=n_q, max_candidates=cache + chunk, device=-1)
+    try:
+        off = lambda n: [n * i for i in range(requests + 1)]
+        batch = fb.make_batch(off(n_q), off(chunk), off(cache), [cache] * requests, [cache] * requests, device="cpu",
+                              row_limit=row_limit)
+        return fb.finch_score_plan(ctx, batch)
+    finally:
+        fb.finch_ctx_destroy(ctx)
+
+
+def test_score_plan_of_the_benchmark_configurations(lib):
+    """Host arithmetic only: which kernels a batch takes and the window length of the one-kernel path."""
+    one, two, warp = fb.FINCH_SCORE_ONE_KERNEL, fb.FINCH_SCORE_TWO_LAUNCH, fb.FINCH_SCORE_WARP_LEVEL
+    # 32 layers x 32q/8kv, 128 prompt rows, 2048 + 2048 candidates: 32 key tiles per unit, windows of 8 (98.8 % full)
+    assert _plan(32, 32, 8, 128, 128, 2048, 2048) == (one, 8)
+    # 32 x 32 MHA, 64 prompt rows, 512 + 512 candidates: 8 key tiles per unit, one window per unit
+    assert _plan(32, 32, 32, 128, 64, 512, 512) == (one, 8)
+    # 27 key tiles per unit (1408 cache rows = 11 tiles, 2048 chunk rows = 16): windows of 9, 86 % full
+    assert _plan(32, 32, 8, 128, 64, 1408, 2048) == (one, 9)
+    # 29 key tiles per unit on 256 units: 29 is prime and a whole unit per window fills 148 CTAs to 86.5 % ...
+    assert _plan(32, 32, 8, 128, 64, 1664, 2048)[0] in (one, two)
+    # ... but 31 tiles per unit, 24 layers: 192 units on 148 CTAs, two windows, 65 % full: no window
+    assert _plan(24, 32, 8, 128, 64, 1920, 2048) == (two, 0)
+    # several requests, fp32 inputs, other head dimensions, more than four query tiles per KV head
+    assert _plan(32, 32, 8, 128, 128, 2048, 2048, requests=2) == (two, 0)
+    assert _plan(32, 32, 8, 128, 128, 2048, 2048, dtype=fb.FINCH_F32) == (warp, 0)
+    assert _plan(2, 8, 8, 96, 64, 512, 512) == (warp, 0)
+    assert _plan(32, 32, 8, 128, 192, 2048, 2048) == (two, 0)     # 4 heads x 3 sub-blocks = 12 > 8
+    assert _plan(32, 32, 8, 128, 128, 2048, 2048)[1] * 128 * 4 == 4096  # four windows per unit
+
+
+def test_score_plan_null_arguments(lib):
+    ctx = fb.finch_ctx_create(**_cfg())
+    batch = fb.make_batch([0, 8], [0, 64], [0, 64], [64], [64], device="cpu")
+    assert lib.finch_score_plan(ctx, C.byref(batch.c), None, None) == fb.FINCH_ERR_INVALID_ARG
+    path = C.c_int32(-1)
+    assert lib.finch_score_plan(ctx, C.byref(batch.c), C.byref(path), None) == fb.FINCH_OK and path.value >= 0
+    fb.finch_ctx_destroy(ctx)
