@@ -95,10 +95,14 @@ class ClockSampler:
         self.proc, self.gpu = None, gpu_index
 
     def start(self):
+        import tempfile
         try:
+            # into a file, not a pipe: nobody reads before stop(), and a full pipe would stall the sampler for the
+            # rest of a long run (its later samples, those of the timed steps, would be missing)
+            self.out = tempfile.TemporaryFile(mode="w+")
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}",
                                           "--format=csv,noheader,nounits", "-lms", "20"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                                         stdout=self.out, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
 
@@ -109,10 +113,13 @@ class ClockSampler:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
         try:
-            out, _ = self.proc.communicate(timeout=5)
+            self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-            out, _ = self.proc.communicate()
+            self.proc.wait()
+        self.out.seek(0)
+        out = self.out.read()
+        self.out.close()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
         rows = []
         for line in out.splitlines():
