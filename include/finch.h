@@ -174,7 +174,8 @@ finch_status finch_score(finch_ctx *ctx, const finch_tensor *prompt_q, const fin
  *  - FINCH_SCORE_ONE_KERNEL: bf16, head_dim 64 or 128, a single request without row_limit, at most four 128-row
  *    query tiles per KV head (queries per KV head x ceil(prompt rows / 64) <= 8), and a window length for its key
  *    tiles exists: a divisor W of the tiles per (layer, KV head) unit with W >= 4 (or the whole unit),
- *    tiles / W <= 8, W x SMs x tile bytes <= 40 MiB, and the persistent grid's CTA x window slots >= 85 % full.
+ *    tiles / W <= 8, the persistent grid's CTA x window slots >= 85 % full, and W x SMs x tile bytes <= 40 MiB
+ *    unless no shorter window qualifies; of several the fullest, longer ones preferred.
  *    *window receives W (key tiles of 128 candidates).  Both sweeps of the softmax run in one persistent kernel.
  *  - FINCH_SCORE_TWO_LAUNCH: bf16, head_dim 64 or 128 otherwise (several requests, causal rows, longer prompts, no
  *    usable window): row statistics and column sums in two tensor-core launches.  *window = 0.
